@@ -1,0 +1,159 @@
+/*
+ * headcast.h - C ABI of the HeadCast attention path for NVIDIA B200 (sm_100a).
+ *
+ * HeadCast (Sec. 4 of the paper) serves the attention layers of an autoregressive video
+ * diffusion transformer that generates a video block by block over a KV cache (Sec. 3.1):
+ *   warm-up with full attention -> one-time head classification (Sec. 4.2, Eq. 2-5) ->
+ *   split of the monolithic cache into per-archetype buffers (Sec. 4.3) ->
+ *   head-specific attention (Sec. 4.4) with a per-block append and roll of those buffers.
+ * One headcast_ctx is one attention layer.  Batch size is 1.
+ *
+ * Conventions for every call:
+ *   - returns HC_OK (0) or a negative HC_ERR_* code; never throws, aborts or prints.
+ *     headcast_last_error() gives a context-owned, human-readable reason for the last failure.
+ *   - tensor arguments named *_dev are DEVICE pointers owned by the caller, 16-byte aligned,
+ *     contiguous, bf16, layout [L][H][d]: L = frames_per_block*grid_h*grid_w tokens of one
+ *     block in (frame, grid row, grid column) order, H = n_heads, d = head_dim.
+ *     arguments named *_host are HOST pointers.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Work is enqueued
+ *     on it and the call returns without waiting, except where a call says it synchronises.
+ *   - the context owns every cache, table and scratch buffer (device memory it allocates at
+ *     headcast_create / headcast_split_cache and frees at headcast_destroy).  The caller must
+ *     keep the context's device current and must not use one context from two threads at once.
+ *   - a kernel that gave up on a bounded wait sets a device status word; the next synchronising
+ *     call, or headcast_check(), reports it as HC_ERR_TIMEOUT.
+ *
+ * States: FILLING (monolithic cache only) --headcast_split_cache--> SPLIT.  A call made in
+ * the wrong state returns HC_ERR_STATE and changes nothing.
+ */
+#ifndef HEADCAST_H_
+#define HEADCAST_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+  HC_OK = 0,
+  HC_ERR_INVALID_ARG = -1,
+  HC_ERR_STATE = -2,
+  HC_ERR_CUDA = -3,
+  HC_ERR_NOMEM = -4,
+  HC_ERR_UNSUPPORTED = -5,
+  HC_ERR_TIMEOUT = -6
+};
+
+/* Head archetypes (Sec. 3.2, Eq. 5). */
+enum { HC_SINK = 0, HC_DUMMY = 1, HC_SPATIAL = 2, HC_GLOBAL = 3 };
+
+/* Per-head score vector written by headcast_classify. */
+enum {
+  HC_SCORE_COS_SINK = 0,    /* Eq. 3, m = sink   */
+  HC_SCORE_COS_DUMMY = 1,   /* Eq. 3, m = dummy  */
+  HC_SCORE_COS_SPATIAL = 2, /* Eq. 3, m = spatial */
+  HC_SCORE_P5_SPATIAL = 3,  /* 5th percentile of the token-wise spatial cosines (Eq. 4) */
+  HC_SCORE_MSE_SPATIAL = 4, /* MSE(O_spatial, O_ref) over all L*d elements (Eq. 4) */
+  HC_SCORE_SCORE = 5,       /* P5 - gamma * MSE (Eq. 4) */
+  HC_SCORE_MASS_FIRST = 6,  /* mean attention mass on the first cached block */
+  HC_SCORE_MASS_LAST = 7,   /* ... on the newest block */
+  HC_SCORE_MASS_SPATIAL = 8,/* ... inside the (2r+1)x(2r+1) neighbourhood, any frame */
+  HC_SCORE_MASS_REST = 9,   /* ... on everything else */
+  HC_N_SCORES = 10
+};
+
+typedef struct headcast_config {
+  int32_t n_heads;          /* H, 1..64 */
+  int32_t head_dim;         /* d, 64 or 128 */
+  int32_t grid_h, grid_w;   /* latent token grid of one frame */
+  int32_t frames_per_block; /* 3 in the paper (Sec. 5.1) */
+  int32_t n_blocks;         /* cache capacity in blocks (2..32), counting the sink block and the newest block */
+  int32_t cell_h, cell_w;   /* deployed Spatial cell, 10 x 10 in the paper (Sec. 5.1) */
+  /* optional explicit cell edges (HOST arrays, copied at create; 0 = first edge, grid = last).
+   * NULL/0 selects the default rule: n = max(1, floor(grid/cell + 1/2)) cells per axis, edge i = floor(i*grid/n). */
+  const int32_t* row_edges_host;
+  int32_t n_row_edges;
+  const int32_t* col_edges_host;
+  int32_t n_col_edges;
+  int32_t proxy_radius;     /* r of the Spatial proxy, 2 in the paper */
+  float theta_sink, theta_dummy, theta_spatial; /* 0.95 each (Sec. 5.1) */
+  float theta_score;        /* 0.755 */
+  float gamma;              /* 5 */
+  float softmax_scale;      /* 0 selects 1/sqrt(d) */
+  int32_t keep_monolithic;  /* nonzero: keep appending to the monolithic cache after the split, so that
+                               headcast_full_attend (the dense baseline) stays usable on the same history */
+} headcast_config;
+
+typedef struct headcast_ctx headcast_ctx;
+
+/* Fills *cfg with the paper's constants (Sec. 5.1); sizes are left zero for the caller. */
+void headcast_default_config(headcast_config* cfg);
+
+/* Validates cfg, allocates the (zeroed) monolithic cache on the current device and returns a context in *out.
+ * Synchronises the device. */
+int headcast_create(const headcast_config* cfg, headcast_ctx** out);
+
+/* Frees everything the context owns.  Synchronises the device.  NULL is accepted. */
+int headcast_destroy(headcast_ctx* ctx);
+
+/* Sec. 3.1 / 4.3: adds one generated block's K and V ([L][H][d] each, device) to the cache.
+ * While the cache is not full the block is placed after the newest one; once full, the oldest block other
+ * than the first (sink) block is evicted.  Before the split this updates the monolithic cache; after it,
+ * the per-archetype buffers: Sink heads keep their frozen first block, Dummy heads overwrite their single
+ * block, Global and Spatial heads slide their window.  Pure byte movement: stored values are bit-identical. */
+int headcast_append(headcast_ctx* ctx, const void* k_new_dev, const void* v_new_dev, void* stream);
+
+/* Dense baseline and warm-up path (Sec. 3.1; "Global Path", Sec. 4.4): every head attends to every cached
+ * token of the monolithic cache.  q_dev and out_dev are [L][H][d] bf16.  Needs at least one cached block;
+ * after the split it needs keep_monolithic. */
+int headcast_full_attend(headcast_ctx* ctx, const void* q_dev, void* out_dev, void* stream);
+
+/* Sec. 4.2: one-time classification with the block's queries q_dev at the maximum-noise step.  Computes the
+ * full-context reference output (Eq. 2) and the Sink, Dummy and Spatial proxy outputs, the mean cosines
+ * (Eq. 3), the Spatial score (Eq. 4) and the label of every head (Eq. 5).  Needs >= 2 cached blocks and
+ * state FILLING.  Synchronises `stream`; writes labels_host[H] and, if not NULL, scores_host[H][HC_N_SCORES];
+ * the labels are also stored in the context. */
+int headcast_classify(headcast_ctx* ctx, const void* q_dev, int32_t* labels_host, float* scores_host, void* stream);
+
+/* Overrides / reads the stored labels (seeded head mixes, ablations).  Host arrays of H int32. State FILLING. */
+int headcast_set_labels(headcast_ctx* ctx, const int32_t* labels_host);
+int headcast_get_labels(const headcast_ctx* ctx, int32_t* labels_host);
+
+/* Sec. 4.3: slices the monolithic cache along the head dimension into the Sink-Dummy buffer (one block per
+ * head), the Global buffer and the Spatial buffer (full window each).  Needs labels and >= 1 cached block.
+ * Allocates the buffers (and frees the monolithic cache unless keep_monolithic).  State becomes SPLIT. */
+int headcast_split_cache(headcast_ctx* ctx, void* stream);
+
+/* Sec. 4.4: head-specific attention of one block's queries, one launch for all pathways.  Sink heads read
+ * their first block, Dummy heads the newest block, Global heads the whole window, Spatial heads the keys of
+ * the query's own grid cell in every cached frame.  out_dev[L][H][d]: every head's rows land at its original
+ * head index (the paper's concatenation along heads).  State SPLIT. */
+int headcast_attend(headcast_ctx* ctx, const void* q_dev, void* out_dev, void* stream);
+
+/* Copies what the cache currently keeps for one head into k_out_dev / v_out_dev ([n_tokens][d] bf16, room for
+ * n_blocks*L rows) in LOGICAL order - oldest kept block first, tokens in (frame, row, column) order - whatever
+ * the private physical layout is.  *n_tokens_host receives the row count.  Either output may be NULL. */
+int headcast_export_cache(headcast_ctx* ctx, int32_t head, void* k_out_dev, void* v_out_dev,
+                          int32_t* n_tokens_host, void* stream);
+
+/* Number of cached blocks (before the split: of the monolithic cache; after: of the sliding window). */
+int headcast_n_filled(const headcast_ctx* ctx);
+
+/* Number of kernels this context has launched so far (bookkeeping for benchmarks). */
+int64_t headcast_launch_count(const headcast_ctx* ctx);
+
+/* Algorithmic FLOPs (4 * L_q * L_k * d per head, Appendix B) of the next headcast_attend (dense = 0) or
+ * headcast_full_attend (dense = 1) with the current cache fill and labels. */
+double headcast_attend_flops(const headcast_ctx* ctx, int32_t dense);
+
+/* Synchronises `stream` and reports a device-side status raised by any earlier kernel of this context
+ * (HC_ERR_TIMEOUT if a bounded wait expired). */
+int headcast_check(headcast_ctx* ctx, void* stream);
+
+const char* headcast_last_error(const headcast_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HEADCAST_H_ */

@@ -1,0 +1,193 @@
+"""ctypes binding of libheadcast.so: argument marshalling only.
+
+Every method mirrors the C entry point of the same name in include/headcast.h; tensors are torch
+CUDA tensors whose ``data_ptr()`` is handed to the library, and the current torch stream is passed
+along.  There is no fallback: if the library is missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Sequence
+
+from . import build as _build
+
+SINK, DUMMY, SPATIAL, GLOBAL = 0, 1, 2, 3
+N_SCORES = 10
+ERRORS = {0: "HC_OK", -1: "HC_ERR_INVALID_ARG", -2: "HC_ERR_STATE", -3: "HC_ERR_CUDA", -4: "HC_ERR_NOMEM",
+          -5: "HC_ERR_UNSUPPORTED", -6: "HC_ERR_TIMEOUT"}
+
+EXPORTS = ("headcast_default_config", "headcast_create", "headcast_destroy", "headcast_append",
+           "headcast_full_attend", "headcast_classify", "headcast_set_labels", "headcast_get_labels",
+           "headcast_split_cache", "headcast_attend", "headcast_export_cache", "headcast_n_filled",
+           "headcast_launch_count", "headcast_attend_flops", "headcast_check", "headcast_last_error")
+
+
+class Config(C.Structure):
+    _fields_ = [("n_heads", C.c_int32), ("head_dim", C.c_int32), ("grid_h", C.c_int32), ("grid_w", C.c_int32),
+                ("frames_per_block", C.c_int32), ("n_blocks", C.c_int32), ("cell_h", C.c_int32),
+                ("cell_w", C.c_int32), ("row_edges_host", C.POINTER(C.c_int32)), ("n_row_edges", C.c_int32),
+                ("col_edges_host", C.POINTER(C.c_int32)), ("n_col_edges", C.c_int32),
+                ("proxy_radius", C.c_int32), ("theta_sink", C.c_float), ("theta_dummy", C.c_float),
+                ("theta_spatial", C.c_float), ("theta_score", C.c_float), ("gamma", C.c_float),
+                ("softmax_scale", C.c_float), ("keep_monolithic", C.c_int32)]
+
+
+class HeadCastError(RuntimeError):
+    def __init__(self, code: int, message: str):
+        super().__init__(f"{ERRORS.get(code, code)}: {message}")
+        self.code = code
+
+
+_lib = None
+
+
+def load_library(path: Optional[str] = None) -> C.CDLL:
+    """Loads (building first if the sources are newer) libheadcast.so and declares the prototypes."""
+    global _lib
+    if _lib is not None and path is None:
+        return _lib
+    lib = C.CDLL(path or _build.build())
+    vp, i32p, f32p = C.c_void_p, C.POINTER(C.c_int32), C.POINTER(C.c_float)
+    lib.headcast_default_config.argtypes = [C.POINTER(Config)]
+    lib.headcast_default_config.restype = None
+    lib.headcast_create.argtypes = [C.POINTER(Config), C.POINTER(vp)]
+    lib.headcast_destroy.argtypes = [vp]
+    lib.headcast_append.argtypes = [vp, vp, vp, vp]
+    lib.headcast_full_attend.argtypes = [vp, vp, vp, vp]
+    lib.headcast_classify.argtypes = [vp, vp, i32p, f32p, vp]
+    lib.headcast_set_labels.argtypes = [vp, i32p]
+    lib.headcast_get_labels.argtypes = [vp, i32p]
+    lib.headcast_split_cache.argtypes = [vp, vp]
+    lib.headcast_attend.argtypes = [vp, vp, vp, vp]
+    lib.headcast_export_cache.argtypes = [vp, C.c_int32, vp, vp, i32p, vp]
+    lib.headcast_n_filled.argtypes = [vp]
+    lib.headcast_launch_count.argtypes = [vp]
+    lib.headcast_launch_count.restype = C.c_int64
+    lib.headcast_attend_flops.argtypes = [vp, C.c_int32]
+    lib.headcast_attend_flops.restype = C.c_double
+    lib.headcast_check.argtypes = [vp, vp]
+    lib.headcast_last_error.argtypes = [vp]
+    lib.headcast_last_error.restype = C.c_char_p
+    if path is None:
+        _lib = lib
+    return lib
+
+
+def default_config(**kw) -> Config:
+    cfg = Config()
+    load_library().headcast_default_config(C.byref(cfg))
+    for k, v in kw.items():
+        setattr(cfg, k, v)
+    return cfg
+
+
+def _stream() -> int:
+    import torch
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _ptr(t) -> int:
+    assert t.is_cuda and t.is_contiguous(), "tensors handed to the library must be contiguous CUDA tensors"
+    return t.data_ptr()
+
+
+class HeadCast:
+    """One attention layer's HeadCast context (wraps headcast_ctx*)."""
+
+    def __init__(self, n_heads: int, head_dim: int, grid_h: int, grid_w: int, n_blocks: int,
+                 frames_per_block: int = 3, cell_h: int = 10, cell_w: int = 10, keep_monolithic: bool = False,
+                 row_edges: Optional[Sequence[int]] = None, col_edges: Optional[Sequence[int]] = None, **overrides):
+        self.lib = load_library()
+        cfg = default_config(n_heads=n_heads, head_dim=head_dim, grid_h=grid_h, grid_w=grid_w, n_blocks=n_blocks,
+                             frames_per_block=frames_per_block, cell_h=cell_h, cell_w=cell_w,
+                             keep_monolithic=int(keep_monolithic), **overrides)
+        keep = []
+        if row_edges is not None:
+            arr = (C.c_int32 * len(row_edges))(*row_edges)
+            keep.append(arr)
+            cfg.row_edges_host, cfg.n_row_edges = arr, len(row_edges)
+        if col_edges is not None:
+            arr = (C.c_int32 * len(col_edges))(*col_edges)
+            keep.append(arr)
+            cfg.col_edges_host, cfg.n_col_edges = arr, len(col_edges)
+        self.cfg = cfg
+        self.n_heads, self.head_dim = n_heads, head_dim
+        self.block_tokens = frames_per_block * grid_h * grid_w
+        self.n_blocks = n_blocks
+        self._ctx = C.c_void_p()
+        rc = self.lib.headcast_create(C.byref(cfg), C.byref(self._ctx))
+        if rc != 0:
+            self._ctx = C.c_void_p()
+            raise HeadCastError(rc, "headcast_create failed")
+
+    @classmethod
+    def from_workload(cls, w, **kw) -> "HeadCast":
+        return cls(w.n_heads, w.head_dim, w.grid_h, w.grid_w, w.n_blocks, w.frames_per_block, w.cell_h, w.cell_w, **kw)
+
+    def _check(self, rc: int) -> None:
+        if rc != 0:
+            raise HeadCastError(rc, self.lib.headcast_last_error(self._ctx).decode())
+
+    def destroy(self) -> None:
+        if self._ctx:
+            self.lib.headcast_destroy(self._ctx)
+            self._ctx = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+    def append(self, k_new, v_new) -> None:
+        self._check(self.lib.headcast_append(self._ctx, _ptr(k_new), _ptr(v_new), _stream()))
+
+    def full_attend(self, q, out) -> None:
+        self._check(self.lib.headcast_full_attend(self._ctx, _ptr(q), _ptr(out), _stream()))
+
+    def classify(self, q):
+        import numpy as np
+        labels = (C.c_int32 * self.n_heads)()
+        scores = (C.c_float * (self.n_heads * N_SCORES))()
+        self._check(self.lib.headcast_classify(self._ctx, _ptr(q), labels, scores, _stream()))
+        return (np.array(labels[:], dtype=np.int32),
+                np.array(scores[:], dtype=np.float32).reshape(self.n_heads, N_SCORES))
+
+    def set_labels(self, labels: Sequence[int]) -> None:
+        arr = (C.c_int32 * self.n_heads)(*[int(v) for v in labels])
+        self._check(self.lib.headcast_set_labels(self._ctx, arr))
+
+    def get_labels(self):
+        arr = (C.c_int32 * self.n_heads)()
+        self._check(self.lib.headcast_get_labels(self._ctx, arr))
+        return list(arr)
+
+    def split_cache(self) -> None:
+        self._check(self.lib.headcast_split_cache(self._ctx, _stream()))
+
+    def attend(self, q, out) -> None:
+        self._check(self.lib.headcast_attend(self._ctx, _ptr(q), _ptr(out), _stream()))
+
+    def export_cache(self, head: int):
+        """Returns (K, V) uint16 CPU arrays [n_tokens, d] of what the cache keeps for ``head``."""
+        import torch
+        n = C.c_int32()
+        k = torch.empty((self.n_blocks * self.block_tokens, self.head_dim), dtype=torch.bfloat16, device="cuda")
+        v = torch.empty_like(k)
+        self._check(self.lib.headcast_export_cache(self._ctx, head, _ptr(k), _ptr(v), C.byref(n), _stream()))
+        torch.cuda.current_stream().synchronize()
+        to_bits = lambda t: t[: n.value].view(torch.int16).cpu().numpy().view("uint16")
+        return to_bits(k), to_bits(v)
+
+    def n_filled(self) -> int:
+        return self.lib.headcast_n_filled(self._ctx)
+
+    def launch_count(self) -> int:
+        return self.lib.headcast_launch_count(self._ctx)
+
+    def attend_flops(self, dense: bool = False) -> float:
+        return self.lib.headcast_attend_flops(self._ctx, int(dense))
+
+    def check(self) -> None:
+        self._check(self.lib.headcast_check(self._ctx, _stream()))

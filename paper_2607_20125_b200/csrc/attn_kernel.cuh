@@ -1,0 +1,465 @@
+// Flash-style attention for every HeadCast pathway on sm_100a tensor cores.
+//
+// One persistent CTA per SM walks a host-built list of work items.  A work item is up to two
+// 128-row query tiles of one head that share one key/value stream:
+//   - S = Q K^T and O += P V run on tcgen05.mma (M = 128, N = 128 / head_dim, bf16 in, fp32 accumulate)
+//     with S, P and O living in tensor memory (P overlays S as packed bf16 and is fed to the second
+//     product straight from tensor memory);
+//   - K/V tiles (128 keys) arrive through TMA into a 2-stage shared-memory ring (128-byte swizzle);
+//   - two softmax warpgroups, one per query tile, own one query row per thread (online softmax in the
+//     exp2 domain, rescaling of O only when the running maximum grew by more than 2^8);
+//   - warp 0 is the TMA producer, warp 1 issues every MMA.
+// Which keys a query tile sees is entirely a property of the work item: a row range of one of the
+// cache buffers (whole window, one block, one Spatial cell) or, for the classification's Spatial
+// proxy, a per-frame band of tokens plus an element-wise neighbourhood test.
+//
+// Every wait is bounded (see mbar_wait); on expiry the CTA drains, frees its tensor memory and leaves,
+// and the host reports HC_ERR_TIMEOUT.
+#pragma once
+#include "tc05.cuh"
+
+namespace hc {
+
+struct CellGeom {
+  int32_t y0, x0, ch, cw;  // top-left grid position and extent of a deployed Spatial cell
+};
+
+enum : int32_t { OUT_BF16 = 0, OUT_PARTIAL = 1, OUT_F32_LSE = 2 };
+
+struct WorkItem {
+  int32_t head;           // original head index: addresses Q and the output
+  int32_t cell;           // < 0: query rows are consecutive tokens; else index into AttnParams::cells
+  int32_t q_start[2];     // first token (cell < 0) or first packed index within the cell's queries
+  int32_t q_count[2];     // valid rows of each 128-row query tile (0: tile unused)
+  int32_t kv_map;         // K map = maps[2 * kv_map], V map = maps[2 * kv_map + 1]
+  int32_t kv_x0;          // element column of this head inside a buffer row
+  int32_t kv_row0;        // buffer row of the first key of segment 0
+  int32_t seg_stride;     // rows between the starts of consecutive segments
+  int32_t seg_len;        // keys per segment
+  int32_t tiles_per_seg;  // ceil(seg_len / 128)
+  int32_t tile_begin;     // this item covers tiles [tile_begin, tile_end) of the segment-major enumeration
+  int32_t tile_end;
+  int32_t out_mode;       // OUT_*
+  int32_t out_slot;       // OUT_PARTIAL: partial slot; OUT_F32_LSE: pass index
+};
+
+struct AttnParams {
+  const WorkItem* items;
+  const int32_t* cta_first;  // [gridDim.x + 1]: CTA b owns items [cta_first[b], cta_first[b + 1])
+  const CUtensorMap* maps;
+  const CellGeom* cells;
+  const __nv_bfloat16* q;  // [L][H][d]
+  __nv_bfloat16* out;      // [L][H][d]
+  float* part_o;           // [slot][256][d] unnormalised partial outputs
+  float2* part_ml;         // [slot][256] (running max in the log2 domain, row sum)
+  float* f32_o;            // [pass][L][H][d] normalised fp32 outputs (classification)
+  float* f32_lse;          // [pass][L][H] natural-log LSE; Spatial proxy also writes [pass + 1] = middle-block LSE
+  int32_t n_heads, tokens_per_frame, grid_w, block_tokens;
+  float scale_log2e;       // softmax scale * log2(e)
+  int32_t* status;
+  // Spatial proxy only
+  int32_t radius;
+  int32_t mid_seg_lo, mid_seg_hi, last_seg_lo, last_seg_hi;  // segments (cached frames) of the middle / newest blocks
+};
+
+constexpr int ATTN_THREADS = 320;  // warp 0: TMA, warp 1: MMA, warps 2-5 / 6-9: softmax for query tile 0 / 1
+constexpr int KV_STAGES = 2;
+constexpr float RESCALE_THRESHOLD = 8.0f;  // log2 units
+
+template <int D>
+struct AttnSmem {
+  static constexpr int BLOCK_BYTES = 128 * 128;      // [128 rows][64 bf16], 128-byte swizzle
+  static constexpr int TILE_BYTES = (D / 64) * BLOCK_BYTES;
+  static constexpr int Q_OFF = 0;
+  static constexpr int K_OFF = 2 * TILE_BYTES;
+  static constexpr int V_OFF = K_OFF + KV_STAGES * TILE_BYTES;
+  static constexpr int TOTAL = V_OFF + KV_STAGES * TILE_BYTES;
+  static constexpr int DYN_BYTES = TOTAL + 1024;  // slack for manual 1024-byte alignment
+};
+
+// Token index of packed query `p` of a cell (frame-major, then cell row, then cell column).
+__device__ __forceinline__ int cell_query_token(const CellGeom& g, int p, int tokens_per_frame, int grid_w) {
+  const int nc = g.ch * g.cw;
+  const int f = p / nc, i = p - f * nc;
+  const int dy = i / g.cw, dx = i - dy * g.cw;
+  return f * tokens_per_frame + (g.y0 + dy) * grid_w + g.x0 + dx;
+}
+
+template <int D, bool PROXY>
+__global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const AttnParams p) {
+  using SM = AttnSmem<D>;
+  constexpr int NB = D / 64;          // 64-column blocks per tile
+  constexpr int QK_STEPS = D / 16;    // k-steps of S = Q K^T
+  constexpr int PV_STEPS = 128 / 16;  // k-steps of O += P V
+  constexpr uint32_t TMEM_COLS = 512;
+  constexpr uint32_t S_COL = 0, O_COL = 256;  // S_t at t*128, O_t at 256 + t*128; P_t overlays S_t
+
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  __shared__ uint64_t bar_q_full[2], bar_s_full[2], bar_p_full[2], bar_o_full[2];
+  __shared__ uint64_t bar_k_full[KV_STAGES], bar_k_free[KV_STAGES], bar_v_full[KV_STAGES], bar_v_free[KV_STAGES];
+  __shared__ uint32_t tmem_slot;
+  __shared__ int abort_flag;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  if (tid == 0) {
+    for (int t = 0; t < 2; ++t) {
+      mbar_init(&bar_q_full[t], 128);
+      mbar_init(&bar_s_full[t], 1);
+      mbar_init(&bar_p_full[t], 128);
+      mbar_init(&bar_o_full[t], 1);
+    }
+    for (int s = 0; s < KV_STAGES; ++s) {
+      mbar_init(&bar_k_full[s], 1);
+      mbar_init(&bar_k_free[s], 1);
+      mbar_init(&bar_v_full[s], 1);
+      mbar_init(&bar_v_free[s], 1);
+    }
+    abort_flag = 0;
+    fence_mbar_init();
+  }
+  if (warp == 1) {
+    tmem_alloc(&tmem_slot, TMEM_COLS);
+    tmem_relinquish();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem = tmem_slot;
+  volatile int* abortp = &abort_flag;
+
+  const int item_lo = p.cta_first[blockIdx.x], item_hi = p.cta_first[blockIdx.x + 1];
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      uint32_t kt = 0;
+      bool ok = true;
+      for (int it = item_lo; it < item_hi && ok; ++it) {
+        const WorkItem w = p.items[it];
+        const CUtensorMap* kmap = &p.maps[2 * w.kv_map];
+        const CUtensorMap* vmap = kmap + 1;
+        for (int tile = w.tile_begin; tile < w.tile_end; ++tile, ++kt) {
+          const int seg = tile / w.tiles_per_seg, c = tile - seg * w.tiles_per_seg;
+          const int row = w.kv_row0 + seg * w.seg_stride + c * 128;
+          const uint32_t st = kt % KV_STAGES, ph = (kt / KV_STAGES) & 1;
+          if (!(ok = mbar_wait(&bar_k_free[st], ph ^ 1, abortp, p.status, 11))) break;
+          mbar_arrive_expect_tx(&bar_k_full[st], SM::TILE_BYTES);
+          for (int b = 0; b < NB; ++b)
+            tma_load_2d(smem + SM::K_OFF + st * SM::TILE_BYTES + b * SM::BLOCK_BYTES, kmap, w.kv_x0 + 64 * b, row,
+                        &bar_k_full[st]);
+          if (!(ok = mbar_wait(&bar_v_free[st], ph ^ 1, abortp, p.status, 12))) break;
+          mbar_arrive_expect_tx(&bar_v_full[st], SM::TILE_BYTES);
+          for (int b = 0; b < NB; ++b)
+            tma_load_2d(smem + SM::V_OFF + st * SM::TILE_BYTES + b * SM::BLOCK_BYTES, vmap, w.kv_x0 + 64 * b, row,
+                        &bar_v_full[st]);
+        }
+      }
+      if (!ok) {
+        // after an expired wait elsewhere: let the copies already in flight land before the CTA leaves
+        for (uint32_t back = 1; back <= KV_STAGES && back <= kt; ++back) {
+          const uint32_t k2 = kt - back, st = k2 % KV_STAGES, ph = (k2 / KV_STAGES) & 1;
+          int local_abort = 0;
+          mbar_wait(&bar_k_full[st], ph, &local_abort, p.status, 13);
+          mbar_wait(&bar_v_full[st], ph, &local_abort, p.status, 13);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      const uint32_t idesc_s = idesc_bf16_f32(128, 128, 0, 0);
+      const uint32_t idesc_o = idesc_bf16_f32(128, D, 0, 1);
+      const uint32_t q_addr = smem_u32(smem + SM::Q_OFF), k_addr = smem_u32(smem + SM::K_OFF),
+                     v_addr = smem_u32(smem + SM::V_OFF);
+      uint32_t kt = 0, q_cnt[2] = {0, 0}, p_cnt[2] = {0, 0};
+      bool ok = true;
+      auto issue_qk = [&](int t, uint32_t st) {
+        for (int kk = 0; kk < QK_STEPS; ++kk) {
+          const uint32_t off = (kk / 4) * SM::BLOCK_BYTES + (kk % 4) * 32;
+          mma_ss(tmem + S_COL + t * 128, smem_desc_sw128(q_addr + t * SM::TILE_BYTES + off, 16, 1024),
+                 smem_desc_sw128(k_addr + st * SM::TILE_BYTES + off, 16, 1024), idesc_s, kk > 0);
+        }
+      };
+      auto issue_pv = [&](int t, uint32_t st, bool accumulate) {
+        for (int kk = 0; kk < PV_STEPS; ++kk)
+          mma_ts(tmem + O_COL + t * 128, tmem + S_COL + t * 128 + kk * 8,
+                 smem_desc_sw128(v_addr + st * SM::TILE_BYTES + kk * 2048, SM::BLOCK_BYTES, 1024), idesc_o,
+                 (accumulate || kk > 0) ? 1u : 0u);
+      };
+      for (int it = item_lo; it < item_hi && ok; ++it) {
+        const WorkItem w = p.items[it];
+        const int nt = w.tile_end - w.tile_begin;
+        const int n_q = w.q_count[1] > 0 ? 2 : 1;
+        {
+          const uint32_t st = kt % KV_STAGES, ph = (kt / KV_STAGES) & 1;
+          if (!(ok = mbar_wait(&bar_k_full[st], ph, abortp, p.status, 21))) break;
+          for (int t = 0; t < n_q && ok; ++t) {
+            if (!(ok = mbar_wait(&bar_q_full[t], q_cnt[t] & 1, abortp, p.status, 22))) break;
+            ++q_cnt[t];
+            tc_fence_after_sync();
+            issue_qk(t, st);
+            mma_commit(&bar_s_full[t]);
+          }
+          if (!ok) break;
+          mma_commit(&bar_k_free[st]);
+        }
+        for (int j = 0; j < nt && ok; ++j) {
+          const uint32_t st = (kt + j) % KV_STAGES, ph = ((kt + j) / KV_STAGES) & 1;
+          const uint32_t st1 = (kt + j + 1) % KV_STAGES, ph1 = ((kt + j + 1) / KV_STAGES) & 1;
+          if (!(ok = mbar_wait(&bar_v_full[st], ph, abortp, p.status, 23))) break;
+          for (int t = 0; t < n_q && ok; ++t) {
+            if (!(ok = mbar_wait(&bar_p_full[t], p_cnt[t] & 1, abortp, p.status, 24))) break;
+            ++p_cnt[t];
+            tc_fence_after_sync();
+            issue_pv(t, st, j > 0);
+            if (j + 1 < nt) {
+              if (t == 0 && !(ok = mbar_wait(&bar_k_full[st1], ph1, abortp, p.status, 25))) break;
+              tc_fence_after_sync();
+              issue_qk(t, st1);
+              mma_commit(&bar_s_full[t]);
+              if (t == n_q - 1) mma_commit(&bar_k_free[st1]);
+            } else {
+              mma_commit(&bar_o_full[t]);
+            }
+          }
+          if (!ok) break;
+          mma_commit(&bar_v_free[st]);
+        }
+        kt += nt;
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ softmax + epilogue warpgroups
+    const int t = (warp - 2) >> 2;                  // query tile of this warpgroup
+    const int r = ((warp & 3) << 5) | lane;         // row inside the tile == TMEM lane
+    const uint32_t lane_off = static_cast<uint32_t>((warp & 3) << 5) << 16;
+    const uint32_t s_addr = tmem + lane_off + S_COL + t * 128;
+    const uint32_t o_addr = tmem + lane_off + O_COL + t * 128;
+    uint8_t* sq = smem + SM::Q_OFF + t * SM::TILE_BYTES;
+    uint32_t s_cnt = 0, o_cnt = 0;
+    bool ok = true;
+    for (int it = item_lo; it < item_hi && ok; ++it) {
+      const WorkItem w = p.items[it];
+      if (w.q_count[t] == 0) continue;
+      const bool row_valid = r < w.q_count[t];
+      int token = 0;
+      if (row_valid) {
+        token = w.q_start[t] + r;
+        if (w.cell >= 0) token = cell_query_token(p.cells[w.cell], token, p.tokens_per_frame, p.grid_w);
+      }
+      // ---- stage this thread's query row into shared memory (swizzled); invalid rows are zero
+      {
+        const uint4* src = reinterpret_cast<const uint4*>(p.q + (static_cast<size_t>(token) * p.n_heads + w.head) * D);
+#pragma unroll
+        for (int c = 0; c < D / 8; ++c) {
+          uint4 v = make_uint4(0, 0, 0, 0);
+          if (row_valid) v = __ldg(src + c);
+          *reinterpret_cast<uint4*>(sq + (c / 8) * SM::BLOCK_BYTES + sw128_offset(r, c % 8)) = v;
+        }
+        fence_proxy_async_smem();
+        tc_fence_before_sync();  // orders this thread's TMEM reads of the previous item before the arrive
+        mbar_arrive(&bar_q_full[t]);
+      }
+      int qy = 0, qx = 0;
+      if (PROXY) {
+        const int pos = token % p.tokens_per_frame;
+        qy = pos / p.grid_w;
+        qx = pos - qy * p.grid_w;
+      }
+      float m_ref = -INFINITY, l_sum = 0.f, l_mid = 0.f;
+      const int nt = w.tile_end - w.tile_begin;
+      for (int j = 0; j < nt; ++j) {
+        const int tile = w.tile_begin + j;
+        const int seg = tile / w.tiles_per_seg, c = tile - seg * w.tiles_per_seg;
+        const int n_valid = min(128, w.seg_len - c * 128);
+        const int tok0 = PROXY ? (w.kv_row0 + c * 128) : 0;  // in-frame token of this tile's first key
+        if (!(ok = mbar_wait(&bar_s_full[t], s_cnt & 1, abortp, p.status, 31))) break;
+        ++s_cnt;
+        tc_fence_after_sync();
+        // pass 1: row maximum of the raw logits
+        float mx = -INFINITY;
+#pragma unroll 1
+        for (int ch = 0; ch < 4; ++ch) {
+          uint32_t v[32];
+          tmem_ld32(s_addr + ch * 32, v);
+          tmem_wait_ld();
+          if (PROXY) {
+            int ky = (tok0 + ch * 32) / p.grid_w, kx = (tok0 + ch * 32) - ky * p.grid_w;
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+              const bool a = (ch * 32 + i < n_valid) && (abs(ky - qy) <= p.radius) && (abs(kx - qx) <= p.radius);
+              if (a) mx = fmaxf(mx, __uint_as_float(v[i]));
+              if (++kx == p.grid_w) { kx = 0; ++ky; }
+            }
+          } else if (ch * 32 + 32 <= n_valid) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(v[i]));
+          } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+              if (ch * 32 + i < n_valid) mx = fmaxf(mx, __uint_as_float(v[i]));
+          }
+        }
+        mx *= p.scale_log2e;  // scale > 0, so the maximum commutes with it
+        // running maximum: move the reference only when some row of the warp outgrew it by 2^8
+        const bool grow = mx > m_ref + RESCALE_THRESHOLD || (m_ref == -INFINITY && mx > -INFINITY);
+        if (__any_sync(0xffffffffu, grow)) {
+          const float m_new = fmaxf(m_ref, mx);
+          const float alpha = (m_new == -INFINITY) ? 1.f : ex2_approx(m_ref - m_new);
+          l_sum *= alpha;
+          l_mid *= alpha;
+          m_ref = m_new;
+          if (j > 0) {  // O_t holds the products of the earlier tiles: bring them to the new reference
+#pragma unroll 1
+            for (int ch = 0; ch < D / 32; ++ch) {
+              uint32_t v[32];
+              tmem_ld32(o_addr + ch * 32, v);
+              tmem_wait_ld();
+#pragma unroll
+              for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(__uint_as_float(v[i]) * alpha);
+              tmem_st32(o_addr + ch * 32, v);
+            }
+          }
+        }
+        const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
+        // pass 2: p = 2^(s * c - m), row sum, bf16 pack into the first 64 columns of S_t
+        float tile_sum = 0.f;
+#pragma unroll 1
+        for (int ch = 0; ch < 4; ++ch) {
+          uint32_t v[32];
+          tmem_ld32(s_addr + ch * 32, v);
+          tmem_wait_ld();
+          float e[32];
+          if (PROXY) {
+            int ky = (tok0 + ch * 32) / p.grid_w, kx = (tok0 + ch * 32) - ky * p.grid_w;
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+              const bool a = (ch * 32 + i < n_valid) && (abs(ky - qy) <= p.radius) && (abs(kx - qx) <= p.radius);
+              e[i] = a ? ex2_approx(fmaf(__uint_as_float(v[i]), p.scale_log2e, -m_use)) : 0.f;
+              if (++kx == p.grid_w) { kx = 0; ++ky; }
+            }
+          } else if (ch * 32 + 32 <= n_valid) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) e[i] = ex2_approx(fmaf(__uint_as_float(v[i]), p.scale_log2e, -m_use));
+          } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+              e[i] = (ch * 32 + i < n_valid) ? ex2_approx(fmaf(__uint_as_float(v[i]), p.scale_log2e, -m_use)) : 0.f;
+          }
+          uint32_t pk[16];
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            tile_sum += e[2 * i] + e[2 * i + 1];
+            pk[i] = pack_bf16x2(e[2 * i], e[2 * i + 1]);
+          }
+          tmem_st16(s_addr + ch * 16, pk);
+        }
+        l_sum += tile_sum;
+        if (PROXY && seg >= p.mid_seg_lo && seg < p.mid_seg_hi && !(seg >= p.last_seg_lo && seg < p.last_seg_hi))
+          l_mid += tile_sum;
+        tmem_wait_st();
+        tc_fence_before_sync();
+        mbar_arrive(&bar_p_full[t]);
+      }
+      if (!ok) break;
+      // ---- epilogue
+      if (!(ok = mbar_wait(&bar_o_full[t], o_cnt & 1, abortp, p.status, 32))) break;
+      ++o_cnt;
+      tc_fence_after_sync();
+      const float inv = (l_sum > 0.f) ? 1.f / l_sum : 0.f;
+      const float mult = (w.out_mode == OUT_PARTIAL) ? 1.f : inv;
+      const size_t row_elem = (static_cast<size_t>(token) * p.n_heads + w.head) * D;
+#pragma unroll 1
+      for (int ch = 0; ch < D / 32; ++ch) {
+        uint32_t v[32];
+        tmem_ld32(o_addr + ch * 32, v);
+        tmem_wait_ld();
+        if (!row_valid) continue;
+        if (w.out_mode == OUT_BF16) {
+          uint4* dst = reinterpret_cast<uint4*>(p.out + row_elem + ch * 32);
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            uint4 o4;
+            o4.x = pack_bf16x2(__uint_as_float(v[8 * i + 0]) * mult, __uint_as_float(v[8 * i + 1]) * mult);
+            o4.y = pack_bf16x2(__uint_as_float(v[8 * i + 2]) * mult, __uint_as_float(v[8 * i + 3]) * mult);
+            o4.z = pack_bf16x2(__uint_as_float(v[8 * i + 4]) * mult, __uint_as_float(v[8 * i + 5]) * mult);
+            o4.w = pack_bf16x2(__uint_as_float(v[8 * i + 6]) * mult, __uint_as_float(v[8 * i + 7]) * mult);
+            dst[i] = o4;
+          }
+        } else {
+          float* base = (w.out_mode == OUT_PARTIAL)
+                            ? p.part_o + (static_cast<size_t>(w.out_slot) * 256 + t * 128 + r) * D
+                            : p.f32_o + static_cast<size_t>(w.out_slot) * p.block_tokens * p.n_heads * D + row_elem;
+          float4* dst = reinterpret_cast<float4*>(base + ch * 32);
+#pragma unroll
+          for (int i = 0; i < 8; ++i)
+            dst[i] = make_float4(__uint_as_float(v[4 * i + 0]) * mult, __uint_as_float(v[4 * i + 1]) * mult,
+                                 __uint_as_float(v[4 * i + 2]) * mult, __uint_as_float(v[4 * i + 3]) * mult);
+        }
+      }
+      if (row_valid) {
+        if (w.out_mode == OUT_PARTIAL) {
+          p.part_ml[static_cast<size_t>(w.out_slot) * 256 + t * 128 + r] = make_float2(m_ref, l_sum);
+        } else if (w.out_mode == OUT_F32_LSE) {
+          const float ln2 = 0.6931471805599453f;
+          const size_t lh = static_cast<size_t>(p.block_tokens) * p.n_heads;
+          const size_t idx = static_cast<size_t>(token) * p.n_heads + w.head;
+          p.f32_lse[w.out_slot * lh + idx] = (l_sum > 0.f) ? m_ref * ln2 + __logf(l_sum) : -INFINITY;
+          if (PROXY) p.f32_lse[(w.out_slot + 1) * lh + idx] = (l_mid > 0.f) ? m_ref * ln2 + __logf(l_mid) : -INFINITY;
+        }
+      }
+    }
+  }
+  // ------------------------------------------------------------------ teardown
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after_sync();
+    tmem_dealloc(tmem, TMEM_COLS);
+  }
+}
+
+// Merges the partial results of query tiles whose key range was cut into several work items:
+// out = sum_i 2^(m_i - m) O_i / sum_i 2^(m_i - m) l_i.  One thread per (row, 8 output columns).
+struct CombineEntry {
+  int32_t head, cell, q_start, q_count;  // one 128-row query tile
+  int32_t first_slot, n_parts, sub;      // partial slots first_slot .. +n_parts-1, rows sub*128 .. of each slot
+  int32_t pad;
+};
+
+template <int D>
+__global__ void combine_kernel(const CombineEntry* entries, const CellGeom* cells, const float* part_o,
+                               const float2* part_ml, __nv_bfloat16* out, int n_heads, int tokens_per_frame,
+                               int grid_w) {
+  const CombineEntry e = entries[blockIdx.x];
+  constexpr int CHUNKS = D / 8;
+  for (int idx = threadIdx.x; idx < e.q_count * CHUNKS; idx += blockDim.x) {
+    const int r = idx / CHUNKS, c = idx - r * CHUNKS;
+    float m = -INFINITY;
+    for (int i = 0; i < e.n_parts; ++i)
+      m = fmaxf(m, part_ml[static_cast<size_t>(e.first_slot + i) * 256 + e.sub * 128 + r].x);
+    float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0}, l = 0.f;
+    for (int i = 0; i < e.n_parts; ++i) {
+      const size_t row = static_cast<size_t>(e.first_slot + i) * 256 + e.sub * 128 + r;
+      const float2 ml = part_ml[row];
+      const float wgt = (ml.x == -INFINITY) ? 0.f : ex2_approx(ml.x - m);
+      l += wgt * ml.y;
+      const float4* src = reinterpret_cast<const float4*>(part_o + row * D + c * 8);
+      const float4 a = src[0], b = src[1];
+      acc[0] += wgt * a.x; acc[1] += wgt * a.y; acc[2] += wgt * a.z; acc[3] += wgt * a.w;
+      acc[4] += wgt * b.x; acc[5] += wgt * b.y; acc[6] += wgt * b.z; acc[7] += wgt * b.w;
+    }
+    const float inv = l > 0.f ? 1.f / l : 0.f;
+    int token = e.q_start + r;
+    if (e.cell >= 0) token = cell_query_token(cells[e.cell], token, tokens_per_frame, grid_w);
+    uint4 o4;
+    o4.x = pack_bf16x2(acc[0] * inv, acc[1] * inv);
+    o4.y = pack_bf16x2(acc[2] * inv, acc[3] * inv);
+    o4.z = pack_bf16x2(acc[4] * inv, acc[5] * inv);
+    o4.w = pack_bf16x2(acc[6] * inv, acc[7] * inv);
+    *reinterpret_cast<uint4*>(out + (static_cast<size_t>(token) * n_heads + e.head) * D + c * 8) = o4;
+  }
+}
+
+}  // namespace hc

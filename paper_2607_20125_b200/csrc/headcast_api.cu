@@ -1,0 +1,892 @@
+// C ABI of the HeadCast attention path (see include/headcast.h): context, state machine, cache ring,
+// tile scheduling, and the launches of the kernels in attn_kernel.cuh / copy_kernels.cuh /
+// score_kernels.cuh.  No CPU fallback exists: every step of the path runs in those kernels.
+#include "../../include/headcast.h"
+
+#include <algorithm>
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <queue>
+#include <string>
+#include <vector>
+
+#include "attn_kernel.cuh"
+#include "copy_kernels.cuh"
+#include "score_kernels.cuh"
+#include "tmap.h"
+
+using namespace hc;
+
+namespace {
+
+enum { STATE_FILLING = 0, STATE_SPLIT = 1 };
+enum { MAP_MONO = 0, MAP_SD = 1, MAP_GLOBAL = 2, MAP_SPATIAL = 3, N_MAP_PAIRS = 4 };
+
+template <typename T>
+struct DevBuf {  // grow-only device array
+  T* ptr = nullptr;
+  size_t cap = 0;
+  cudaError_t reserve(size_t n) {
+    if (n <= cap) return cudaSuccess;
+    if (ptr) cudaFree(ptr);
+    ptr = nullptr;
+    cap = 0;
+    cudaError_t e = cudaMalloc(&ptr, n * sizeof(T));
+    if (e == cudaSuccess) cap = n;
+    return e;
+  }
+  void release() {
+    if (ptr) cudaFree(ptr);
+    ptr = nullptr;
+    cap = 0;
+  }
+};
+
+struct Schedule {
+  int key_filled = -1;  // cache fill the lists were built for
+  std::vector<WorkItem> items;
+  std::vector<int32_t> cta_first;
+  std::vector<CombineEntry> combine;
+  DevBuf<WorkItem> items_dev;
+  DevBuf<int32_t> cta_first_dev;
+  DevBuf<CombineEntry> combine_dev;
+  int n_slots = 0;
+  bool uploaded = false;
+  double flops = 0.0;
+  void release() {
+    items_dev.release();
+    cta_first_dev.release();
+    combine_dev.release();
+  }
+};
+
+}  // namespace
+
+struct headcast_ctx {
+  headcast_config cfg;
+  int H, D, L, T_f, F_b, n_blk, CH, G_h, G_w;
+  float scale;
+  int state = STATE_FILLING;
+  std::vector<int> slots;  // logical block -> physical ring slot (index 0 = sink block)
+  bool have_labels = false;
+  std::vector<int32_t> labels;
+  int n_cls[4] = {0, 0, 0, 0};
+  int8_t cls[MAX_HEADS], idx[MAX_HEADS];
+  std::vector<int> row_edges, col_edges;
+  std::vector<CellGeom> cells;
+  std::vector<int> cell_tok_off;  // tokens per frame in earlier cells
+
+  __nv_bfloat16 *mono_k = nullptr, *mono_v = nullptr;
+  __nv_bfloat16 *sd_k = nullptr, *sd_v = nullptr, *g_k = nullptr, *g_v = nullptr, *sp_k = nullptr, *sp_v = nullptr;
+  int32_t *sp_base = nullptr, *sp_nc = nullptr;
+  CellGeom* cells_dev = nullptr;
+  CUtensorMap* maps_dev = nullptr;
+  int32_t* status_dev = nullptr;
+
+  Schedule sched_dense, sched_hc, sched_cls, sched_proxy;
+  DevBuf<float> part_o;
+  DevBuf<float2> part_ml;
+  DevBuf<float> cls_o, cls_lse, cls_tok, cls_scores;
+  DevBuf<int32_t> cls_labels;
+
+  int n_sm = 148;
+  int64_t launches = 0;
+  std::string err;
+};
+
+namespace {
+
+int fail(headcast_ctx* c, int code, const char* fmt, ...) {
+  if (c) {
+    char buf[512];
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(buf, sizeof(buf), fmt, ap);
+    va_end(ap);
+    c->err = buf;
+  }
+  return code;
+}
+
+#define HC_CUDA(c, expr)                                                                           \
+  do {                                                                                             \
+    cudaError_t e_ = (expr);                                                                       \
+    if (e_ != cudaSuccess)                                                                         \
+      return fail((c), e_ == cudaErrorMemoryAllocation ? HC_ERR_NOMEM : HC_ERR_CUDA, "%s: %s", #expr, \
+                  cudaGetErrorString(e_));                                                         \
+  } while (0)
+
+std::vector<int> default_edges(int grid, int cell) {
+  const int n = std::max(1, static_cast<int>(std::floor(static_cast<double>(grid) / cell + 0.5)));
+  std::vector<int> e(n + 1);
+  for (int i = 0; i <= n; ++i) e[i] = static_cast<int>((static_cast<long long>(i) * grid) / n);
+  return e;
+}
+
+bool edges_ok(const std::vector<int>& e, int grid) {
+  if (e.size() < 2 || e.front() != 0 || e.back() != grid) return false;
+  for (size_t i = 1; i < e.size(); ++i)
+    if (e[i] <= e[i - 1]) return false;
+  return true;
+}
+
+bool aligned16(const void* p) { return p != nullptr && (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+size_t cache_elems(const headcast_ctx* c, int heads) {
+  return static_cast<size_t>(heads) * c->n_blk * c->L * c->D;
+}
+
+// ---------------------------------------------------------------------------------- tensor maps
+int build_maps(headcast_ctx* c) {
+  CUtensorMap maps[2 * N_MAP_PAIRS];
+  std::memset(maps, 0, sizeof(maps));
+  const uint64_t win_rows = static_cast<uint64_t>(c->n_blk) * c->L;
+  bool ok = true;
+  if (c->mono_k) {
+    ok = ok && make_tmap_bf16_2d(&maps[2 * MAP_MONO], c->mono_k, static_cast<uint64_t>(c->H) * c->D, win_rows,
+                                 static_cast<uint64_t>(c->H) * c->D, 128);
+    ok = ok && make_tmap_bf16_2d(&maps[2 * MAP_MONO + 1], c->mono_v, static_cast<uint64_t>(c->H) * c->D, win_rows,
+                                 static_cast<uint64_t>(c->H) * c->D, 128);
+  }
+  if (c->sd_k) {
+    const uint64_t rows = static_cast<uint64_t>(c->n_cls[CLS_SINK] + c->n_cls[CLS_DUMMY]) * c->L;
+    ok = ok && make_tmap_bf16_2d(&maps[2 * MAP_SD], c->sd_k, c->D, rows, c->D, 128);
+    ok = ok && make_tmap_bf16_2d(&maps[2 * MAP_SD + 1], c->sd_v, c->D, rows, c->D, 128);
+  }
+  if (c->g_k) {
+    const uint64_t rows = c->n_cls[CLS_GLOBAL] * win_rows;
+    ok = ok && make_tmap_bf16_2d(&maps[2 * MAP_GLOBAL], c->g_k, c->D, rows, c->D, 128);
+    ok = ok && make_tmap_bf16_2d(&maps[2 * MAP_GLOBAL + 1], c->g_v, c->D, rows, c->D, 128);
+  }
+  if (c->sp_k) {
+    const uint64_t rows = c->n_cls[CLS_SPATIAL] * win_rows;
+    ok = ok && make_tmap_bf16_2d(&maps[2 * MAP_SPATIAL], c->sp_k, c->D, rows, c->D, 128);
+    ok = ok && make_tmap_bf16_2d(&maps[2 * MAP_SPATIAL + 1], c->sp_v, c->D, rows, c->D, 128);
+  }
+  if (!ok) return fail(c, HC_ERR_CUDA, "cuTensorMapEncodeTiled failed or is unavailable");
+  HC_CUDA(c, cudaMemcpy(c->maps_dev, maps, sizeof(maps), cudaMemcpyHostToDevice));
+  return HC_OK;
+}
+
+// ---------------------------------------------------------------------------------- scheduling
+struct Proto {  // one (head, query-tile pair, key range) before it is cut into parts
+  WorkItem w;
+  int n_tiles;
+};
+
+void add_query_pairs(std::vector<Proto>& out, WorkItem base, int n_queries, int n_tiles) {
+  for (int q0 = 0; q0 < n_queries; q0 += 256) {
+    Proto p;
+    p.w = base;
+    p.w.q_start[0] = q0;
+    p.w.q_start[1] = q0 + 128;
+    p.w.q_count[0] = std::min(128, n_queries - q0);
+    p.w.q_count[1] = std::max(0, std::min(128, n_queries - q0 - 128));
+    p.w.tile_begin = 0;
+    p.w.tile_end = n_tiles;
+    p.n_tiles = n_tiles;
+    out.push_back(p);
+  }
+}
+
+WorkItem range_item(int head, int map, int x0, long long row0, int n_keys) {
+  WorkItem w;
+  std::memset(&w, 0, sizeof(w));
+  w.head = head;
+  w.cell = -1;
+  w.kv_map = map;
+  w.kv_x0 = x0;
+  w.kv_row0 = static_cast<int32_t>(row0);
+  w.seg_stride = 0;
+  w.seg_len = n_keys;
+  w.tiles_per_seg = (n_keys + 127) / 128;
+  w.out_mode = OUT_BF16;
+  return w;
+}
+
+constexpr double ITEM_OVERHEAD = 3.0;  // tile-times charged per item for the query load, pipeline fill and epilogue
+
+double item_cost(const WorkItem& w) {
+  const int n_q = w.q_count[1] > 0 ? 2 : 1;
+  return static_cast<double>(n_q) * (w.tile_end - w.tile_begin) + ITEM_OVERHEAD;
+}
+
+// Cuts long items along the key range (partials merged by combine_kernel), then assigns items to CTAs
+// longest-first onto the least loaded CTA.
+void finalize_schedule(headcast_ctx* c, Schedule& s, std::vector<Proto>& protos, bool allow_split) {
+  s.items.clear();
+  s.combine.clear();
+  s.n_slots = 0;
+  double total = 0.0;
+  for (const Proto& p : protos) total += item_cost(p.w);
+  const double max_cost = std::max(48.0, total / c->n_sm / 2.5);
+  std::vector<WorkItem> all;
+  for (const Proto& p : protos) {
+    const int n_q = p.w.q_count[1] > 0 ? 2 : 1;
+    int parts = 1;
+    if (allow_split) parts = std::max(1, static_cast<int>(std::ceil(item_cost(p.w) / max_cost)));
+    parts = std::min(parts, p.n_tiles);
+    if (parts == 1) {
+      all.push_back(p.w);
+      continue;
+    }
+    const int per = (p.n_tiles + parts - 1) / parts;
+    const int first_slot = s.n_slots;
+    int made = 0;
+    for (int b = 0; b < p.n_tiles; b += per, ++made) {
+      WorkItem w = p.w;
+      w.tile_begin = b;
+      w.tile_end = std::min(p.n_tiles, b + per);
+      w.out_mode = OUT_PARTIAL;
+      w.out_slot = s.n_slots++;
+      all.push_back(w);
+    }
+    for (int t = 0; t < n_q; ++t) {
+      CombineEntry e;
+      e.head = p.w.head;
+      e.cell = p.w.cell;
+      e.q_start = p.w.q_start[t];
+      e.q_count = p.w.q_count[t];
+      e.first_slot = first_slot;
+      e.n_parts = made;
+      e.sub = t;
+      e.pad = 0;
+      s.combine.push_back(e);
+    }
+  }
+  std::stable_sort(all.begin(), all.end(), [](const WorkItem& a, const WorkItem& b) { return item_cost(a) > item_cost(b); });
+  const int n_cta = c->n_sm;
+  std::vector<std::vector<WorkItem>> bins(n_cta);
+  typedef std::pair<double, int> Load;
+  std::priority_queue<Load, std::vector<Load>, std::greater<Load>> pq;
+  for (int b = 0; b < n_cta; ++b) pq.push(Load(0.0, b));
+  for (const WorkItem& w : all) {
+    Load l = pq.top();
+    pq.pop();
+    bins[l.second].push_back(w);
+    pq.push(Load(l.first + item_cost(w), l.second));
+  }
+  s.cta_first.assign(n_cta + 1, 0);
+  for (int b = 0; b < n_cta; ++b) {
+    s.cta_first[b] = static_cast<int32_t>(s.items.size());
+    s.items.insert(s.items.end(), bins[b].begin(), bins[b].end());
+  }
+  s.cta_first[n_cta] = static_cast<int32_t>(s.items.size());
+  s.uploaded = false;
+}
+
+int n_filled(const headcast_ctx* c) { return static_cast<int>(c->slots.size()); }
+
+void build_dense_schedule(headcast_ctx* c, Schedule& s, int out_mode, bool allow_split) {
+  std::vector<Proto> protos;
+  const int n_keys = n_filled(c) * c->L;
+  for (int h = 0; h < c->H; ++h) {
+    WorkItem w = range_item(h, MAP_MONO, h * c->D, 0, n_keys);
+    w.out_mode = out_mode;
+    add_query_pairs(protos, w, c->L, w.tiles_per_seg);
+  }
+  s.flops = 4.0 * c->H * static_cast<double>(c->L) * n_keys * c->D;
+  finalize_schedule(c, s, protos, allow_split);
+  s.key_filled = n_filled(c);
+}
+
+void build_headcast_schedule(headcast_ctx* c, Schedule& s) {
+  std::vector<Proto> protos;
+  const int nf = n_filled(c);
+  const long long win = static_cast<long long>(c->n_blk) * c->L;
+  double flops = 0.0;
+  for (int h = 0; h < c->H; ++h) {
+    const int cl = c->cls[h], ix = c->idx[h];
+    if (cl == CLS_SINK || cl == CLS_DUMMY) {
+      const int j = (cl == CLS_SINK) ? ix : c->n_cls[CLS_SINK] + ix;
+      WorkItem w = range_item(h, MAP_SD, 0, static_cast<long long>(j) * c->L, c->L);
+      add_query_pairs(protos, w, c->L, w.tiles_per_seg);
+      flops += 4.0 * c->L * static_cast<double>(c->L) * c->D;
+    } else if (cl == CLS_GLOBAL) {
+      WorkItem w = range_item(h, MAP_GLOBAL, 0, ix * win, nf * c->L);
+      add_query_pairs(protos, w, c->L, w.tiles_per_seg);
+      flops += 4.0 * c->L * static_cast<double>(nf) * c->L * c->D;
+    } else {
+      for (size_t ci = 0; ci < c->cells.size(); ++ci) {
+        const int nc = c->cells[ci].ch * c->cells[ci].cw;
+        const long long row0 = ix * win + static_cast<long long>(c->n_blk) * c->F_b * c->cell_tok_off[ci];
+        WorkItem w = range_item(h, MAP_SPATIAL, 0, row0, nf * c->F_b * nc);
+        w.cell = static_cast<int32_t>(ci);
+        add_query_pairs(protos, w, c->F_b * nc, w.tiles_per_seg);
+        flops += 4.0 * (c->F_b * nc) * static_cast<double>(nf * c->F_b * nc) * c->D;
+      }
+    }
+  }
+  s.flops = flops;
+  finalize_schedule(c, s, protos, true);
+  s.key_filled = nf;
+}
+
+int upload_schedule(headcast_ctx* c, Schedule& s, cudaStream_t st) {
+  if (s.uploaded) return HC_OK;
+  HC_CUDA(c, s.items_dev.reserve(std::max<size_t>(1, s.items.size())));
+  HC_CUDA(c, s.cta_first_dev.reserve(s.cta_first.size()));
+  HC_CUDA(c, s.combine_dev.reserve(std::max<size_t>(1, s.combine.size())));
+  if (!s.items.empty())
+    HC_CUDA(c, cudaMemcpyAsync(s.items_dev.ptr, s.items.data(), s.items.size() * sizeof(WorkItem),
+                               cudaMemcpyHostToDevice, st));
+  HC_CUDA(c, cudaMemcpyAsync(s.cta_first_dev.ptr, s.cta_first.data(), s.cta_first.size() * sizeof(int32_t),
+                             cudaMemcpyHostToDevice, st));
+  if (!s.combine.empty())
+    HC_CUDA(c, cudaMemcpyAsync(s.combine_dev.ptr, s.combine.data(), s.combine.size() * sizeof(CombineEntry),
+                               cudaMemcpyHostToDevice, st));
+  if (s.n_slots > 0) {
+    HC_CUDA(c, c->part_o.reserve(static_cast<size_t>(s.n_slots) * 256 * c->D));
+    HC_CUDA(c, c->part_ml.reserve(static_cast<size_t>(s.n_slots) * 256));
+  }
+  s.uploaded = true;
+  return HC_OK;
+}
+
+template <int D, bool PROXY>
+int launch_attn_t(headcast_ctx* c, const AttnParams& p, cudaStream_t st) {
+  static bool configured = false;
+  if (!configured) {
+    HC_CUDA(c, cudaFuncSetAttribute(attn_kernel<D, PROXY>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    AttnSmem<D>::DYN_BYTES));
+    configured = true;
+  }
+  attn_kernel<D, PROXY><<<c->n_sm, ATTN_THREADS, AttnSmem<D>::DYN_BYTES, st>>>(p);
+  HC_CUDA(c, cudaGetLastError());
+  ++c->launches;
+  return HC_OK;
+}
+
+int run_schedule(headcast_ctx* c, Schedule& s, const void* q, void* out, bool proxy, cudaStream_t st) {
+  int rc = upload_schedule(c, s, st);
+  if (rc != HC_OK) return rc;
+  if (s.items.empty()) return HC_OK;
+  AttnParams p;
+  std::memset(&p, 0, sizeof(p));
+  p.items = s.items_dev.ptr;
+  p.cta_first = s.cta_first_dev.ptr;
+  p.maps = c->maps_dev;
+  p.cells = c->cells_dev;
+  p.q = static_cast<const __nv_bfloat16*>(q);
+  p.out = static_cast<__nv_bfloat16*>(out);
+  p.part_o = c->part_o.ptr;
+  p.part_ml = c->part_ml.ptr;
+  p.f32_o = c->cls_o.ptr;
+  p.f32_lse = c->cls_lse.ptr;
+  p.n_heads = c->H;
+  p.tokens_per_frame = c->T_f;
+  p.grid_w = c->G_w;
+  p.block_tokens = c->L;
+  p.scale_log2e = c->scale * 1.4426950408889634f;
+  p.status = c->status_dev;
+  p.radius = c->cfg.proxy_radius;
+  if (proxy) {
+    const int newest = c->slots.back();
+    p.mid_seg_lo = c->F_b;
+    p.mid_seg_hi = n_filled(c) * c->F_b;
+    p.last_seg_lo = newest * c->F_b;
+    p.last_seg_hi = (newest + 1) * c->F_b;
+  }
+  if (c->D == 128)
+    rc = proxy ? launch_attn_t<128, true>(c, p, st) : launch_attn_t<128, false>(c, p, st);
+  else
+    rc = proxy ? launch_attn_t<64, true>(c, p, st) : launch_attn_t<64, false>(c, p, st);
+  if (rc != HC_OK) return rc;
+  if (!s.combine.empty()) {
+    if (c->D == 128)
+      combine_kernel<128><<<static_cast<unsigned>(s.combine.size()), 256, 0, st>>>(
+          s.combine_dev.ptr, c->cells_dev, c->part_o.ptr, c->part_ml.ptr, p.out, c->H, c->T_f, c->G_w);
+    else
+      combine_kernel<64><<<static_cast<unsigned>(s.combine.size()), 256, 0, st>>>(
+          s.combine_dev.ptr, c->cells_dev, c->part_o.ptr, c->part_ml.ptr, p.out, c->H, c->T_f, c->G_w);
+    HC_CUDA(c, cudaGetLastError());
+    ++c->launches;
+  }
+  return HC_OK;
+}
+
+void fill_route(headcast_ctx* c, RouteParams& r) {
+  std::memset(&r, 0, sizeof(r));
+  r.mono_k = reinterpret_cast<uint4*>(c->mono_k);
+  r.mono_v = reinterpret_cast<uint4*>(c->mono_v);
+  r.sd_k = reinterpret_cast<uint4*>(c->sd_k);
+  r.sd_v = reinterpret_cast<uint4*>(c->sd_v);
+  r.g_k = reinterpret_cast<uint4*>(c->g_k);
+  r.g_v = reinterpret_cast<uint4*>(c->g_v);
+  r.sp_k = reinterpret_cast<uint4*>(c->sp_k);
+  r.sp_v = reinterpret_cast<uint4*>(c->sp_v);
+  r.sp_base = c->sp_base;
+  r.sp_nc = c->sp_nc;
+  r.L = c->L;
+  r.H = c->H;
+  r.chunks = c->CH;
+  r.tokens_per_frame = c->T_f;
+  r.frames_per_block = c->F_b;
+  r.n_blocks = c->n_blk;
+  r.n_sink = c->n_cls[CLS_SINK];
+  for (int h = 0; h < c->H; ++h) {
+    r.cls[h] = (c->state == STATE_SPLIT || c->sd_k || c->g_k || c->sp_k) ? c->cls[h] : static_cast<int8_t>(CLS_NONE);
+    r.idx[h] = c->idx[h];
+  }
+}
+
+int launch_route(headcast_ctx* c, const RouteParams& r, cudaStream_t st) {
+  const long long total = static_cast<long long>(r.L) * r.H * r.chunks;
+  const long long per_block = 256LL * ROUTE_UNROLL;
+  const int blocks = static_cast<int>(std::min<long long>((total + per_block - 1) / per_block, c->n_sm * 8LL));
+  route_block_kernel<<<std::max(1, blocks), 256, 0, st>>>(r);
+  HC_CUDA(c, cudaGetLastError());
+  ++c->launches;
+  return HC_OK;
+}
+
+int read_status(headcast_ctx* c, cudaStream_t st) {
+  int32_t status = 0;
+  HC_CUDA(c, cudaMemcpyAsync(&status, c->status_dev, sizeof(status), cudaMemcpyDeviceToHost, st));
+  HC_CUDA(c, cudaStreamSynchronize(st));
+  if (status != 0) {
+    cudaMemsetAsync(c->status_dev, 0, sizeof(int32_t), st);
+    return fail(c, HC_ERR_TIMEOUT, "a kernel gave up on a bounded wait (site %d)", status);
+  }
+  return HC_OK;
+}
+
+void assign_classes(headcast_ctx* c) {
+  for (int k = 0; k < 4; ++k) c->n_cls[k] = 0;
+  for (int h = 0; h < c->H; ++h) {
+    c->cls[h] = static_cast<int8_t>(c->labels[h]);
+    c->idx[h] = static_cast<int8_t>(c->n_cls[c->labels[h]]++);
+  }
+}
+
+}  // namespace
+
+// =====================================================================================================
+extern "C" {
+
+void headcast_default_config(headcast_config* cfg) {
+  if (!cfg) return;
+  std::memset(cfg, 0, sizeof(*cfg));
+  cfg->frames_per_block = 3;
+  cfg->cell_h = 10;
+  cfg->cell_w = 10;
+  cfg->proxy_radius = 2;
+  cfg->theta_sink = cfg->theta_dummy = cfg->theta_spatial = 0.95f;
+  cfg->theta_score = 0.755f;
+  cfg->gamma = 5.0f;
+  cfg->softmax_scale = 0.0f;
+}
+
+int headcast_create(const headcast_config* cfg, headcast_ctx** out) {
+  if (!cfg || !out) return HC_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (cfg->n_heads < 1 || cfg->n_heads > MAX_HEADS || (cfg->head_dim != 64 && cfg->head_dim != 128) ||
+      cfg->grid_h < 1 || cfg->grid_w < 1 || cfg->frames_per_block < 1 || cfg->n_blocks < 2 ||
+      cfg->n_blocks > MAX_BLOCKS || cfg->cell_h < 1 || cfg->cell_w < 1 || cfg->proxy_radius < 0 ||
+      !(cfg->softmax_scale >= 0.0f))
+    return HC_ERR_INVALID_ARG;
+  const long long L = static_cast<long long>(cfg->frames_per_block) * cfg->grid_h * cfg->grid_w;
+  if (L * cfg->n_blocks * cfg->n_heads * cfg->head_dim >= (1LL << 40) || L * cfg->n_blocks * cfg->n_heads >= (1LL << 31))
+    return HC_ERR_INVALID_ARG;
+  headcast_ctx* c = new (std::nothrow) headcast_ctx();
+  if (!c) return HC_ERR_NOMEM;
+  c->cfg = *cfg;
+  c->H = cfg->n_heads;
+  c->D = cfg->head_dim;
+  c->G_h = cfg->grid_h;
+  c->G_w = cfg->grid_w;
+  c->F_b = cfg->frames_per_block;
+  c->T_f = cfg->grid_h * cfg->grid_w;
+  c->L = static_cast<int>(L);
+  c->n_blk = cfg->n_blocks;
+  c->CH = c->D / 8;
+  c->scale = cfg->softmax_scale > 0.f ? cfg->softmax_scale : 1.0f / std::sqrt(static_cast<float>(c->D));
+  c->row_edges = (cfg->row_edges_host && cfg->n_row_edges > 0)
+                     ? std::vector<int>(cfg->row_edges_host, cfg->row_edges_host + cfg->n_row_edges)
+                     : default_edges(c->G_h, cfg->cell_h);
+  c->col_edges = (cfg->col_edges_host && cfg->n_col_edges > 0)
+                     ? std::vector<int>(cfg->col_edges_host, cfg->col_edges_host + cfg->n_col_edges)
+                     : default_edges(c->G_w, cfg->cell_w);
+  c->cfg.row_edges_host = c->cfg.col_edges_host = nullptr;
+  if (!edges_ok(c->row_edges, c->G_h) || !edges_ok(c->col_edges, c->G_w)) {
+    delete c;
+    return HC_ERR_INVALID_ARG;
+  }
+  c->labels.assign(c->H, HC_GLOBAL);
+  for (int h = 0; h < c->H; ++h) {
+    c->cls[h] = CLS_NONE;
+    c->idx[h] = 0;
+  }
+  // deployed cells and the cell-major token order of the Spatial buffers
+  std::vector<int32_t> sp_base(c->T_f), sp_nc(c->T_f);
+  int tok_off = 0;
+  for (size_t i = 0; i + 1 < c->row_edges.size(); ++i)
+    for (size_t j = 0; j + 1 < c->col_edges.size(); ++j) {
+      CellGeom g = {c->row_edges[i], c->col_edges[j], c->row_edges[i + 1] - c->row_edges[i],
+                    c->col_edges[j + 1] - c->col_edges[j]};
+      c->cells.push_back(g);
+      c->cell_tok_off.push_back(tok_off);
+      for (int dy = 0; dy < g.ch; ++dy)
+        for (int dx = 0; dx < g.cw; ++dx) {
+          const int pos = (g.y0 + dy) * c->G_w + g.x0 + dx;
+          sp_base[pos] = c->n_blk * c->F_b * tok_off + dy * g.cw + dx;
+          sp_nc[pos] = g.ch * g.cw;
+        }
+      tok_off += g.ch * g.cw;
+    }
+  int dev = 0;
+  cudaDeviceProp prop;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess) {
+    delete c;
+    return HC_ERR_CUDA;
+  }
+  if (prop.major != 10) {
+    delete c;
+    return HC_ERR_UNSUPPORTED;
+  }
+  c->n_sm = prop.multiProcessorCount;
+  const size_t mono_bytes = cache_elems(c, c->H) * sizeof(__nv_bfloat16);
+  cudaError_t e = cudaSuccess;
+  auto step = [&](cudaError_t r) { if (e == cudaSuccess) e = r; };
+  step(cudaMalloc(&c->mono_k, mono_bytes));
+  step(cudaMalloc(&c->mono_v, mono_bytes));
+  step(cudaMalloc(&c->sp_base, c->T_f * sizeof(int32_t)));
+  step(cudaMalloc(&c->sp_nc, c->T_f * sizeof(int32_t)));
+  step(cudaMalloc(&c->cells_dev, c->cells.size() * sizeof(CellGeom)));
+  step(cudaMalloc(&c->maps_dev, 2 * N_MAP_PAIRS * sizeof(CUtensorMap)));
+  step(cudaMalloc(&c->status_dev, sizeof(int32_t)));
+  if (e == cudaSuccess) {
+    step(cudaMemset(c->mono_k, 0, mono_bytes));
+    step(cudaMemset(c->mono_v, 0, mono_bytes));
+    step(cudaMemset(c->status_dev, 0, sizeof(int32_t)));
+    step(cudaMemcpy(c->sp_base, sp_base.data(), c->T_f * sizeof(int32_t), cudaMemcpyHostToDevice));
+    step(cudaMemcpy(c->sp_nc, sp_nc.data(), c->T_f * sizeof(int32_t), cudaMemcpyHostToDevice));
+    step(cudaMemcpy(c->cells_dev, c->cells.data(), c->cells.size() * sizeof(CellGeom), cudaMemcpyHostToDevice));
+  }
+  int rc = HC_OK;
+  if (e != cudaSuccess) rc = (e == cudaErrorMemoryAllocation) ? HC_ERR_NOMEM : HC_ERR_CUDA;
+  if (rc == HC_OK) rc = build_maps(c);
+  if (rc == HC_OK && cudaDeviceSynchronize() != cudaSuccess) rc = HC_ERR_CUDA;
+  if (rc != HC_OK) {
+    headcast_destroy(c);
+    return rc;
+  }
+  *out = c;
+  return HC_OK;
+}
+
+int headcast_destroy(headcast_ctx* c) {
+  if (!c) return HC_OK;
+  cudaDeviceSynchronize();
+  void* ptrs[] = {c->mono_k, c->mono_v, c->sd_k, c->sd_v, c->g_k, c->g_v, c->sp_k, c->sp_v,
+                  c->sp_base, c->sp_nc, c->cells_dev, c->maps_dev, c->status_dev};
+  for (void* p : ptrs)
+    if (p) cudaFree(p);
+  c->sched_dense.release();
+  c->sched_hc.release();
+  c->sched_cls.release();
+  c->sched_proxy.release();
+  c->part_o.release();
+  c->part_ml.release();
+  c->cls_o.release();
+  c->cls_lse.release();
+  c->cls_tok.release();
+  c->cls_scores.release();
+  c->cls_labels.release();
+  delete c;
+  return HC_OK;
+}
+
+int headcast_append(headcast_ctx* c, const void* k_new, const void* v_new, void* stream) {
+  if (!c) return HC_ERR_INVALID_ARG;
+  if (!aligned16(k_new) || !aligned16(v_new)) return fail(c, HC_ERR_INVALID_ARG, "k_new/v_new must be 16-byte aligned device pointers");
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // ring bookkeeping: the sink block never moves; when full, the oldest rolling block's slot is reused
+  int slot;
+  std::vector<int> next = c->slots;
+  if (static_cast<int>(next.size()) < c->n_blk) {
+    slot = static_cast<int>(next.size());
+    next.push_back(slot);
+  } else if (c->n_blk == 1) {
+    slot = 0;
+  } else {
+    slot = next[1];
+    next.erase(next.begin() + 1);
+    next.push_back(slot);
+  }
+  RouteParams r;
+  fill_route(c, r);
+  r.src_k = static_cast<const uint4*>(k_new);
+  r.src_v = static_cast<const uint4*>(v_new);
+  r.slot = slot;
+  r.copy_mono = c->mono_k != nullptr;
+  r.copy_sink = 0;  // frozen
+  r.copy_dummy = c->state == STATE_SPLIT;
+  r.copy_window = c->state == STATE_SPLIT;
+  int rc = launch_route(c, r, st);
+  if (rc != HC_OK) return rc;
+  c->slots.swap(next);
+  return HC_OK;
+}
+
+int headcast_full_attend(headcast_ctx* c, const void* q, void* out, void* stream) {
+  if (!c) return HC_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(out)) return fail(c, HC_ERR_INVALID_ARG, "q/out must be 16-byte aligned device pointers");
+  if (!c->mono_k) return fail(c, HC_ERR_STATE, "the monolithic cache was released at the split (keep_monolithic = 0)");
+  if (c->slots.empty()) return fail(c, HC_ERR_STATE, "the cache is empty");
+  if (c->sched_dense.key_filled != n_filled(c)) build_dense_schedule(c, c->sched_dense, OUT_BF16, true);
+  return run_schedule(c, c->sched_dense, q, out, false, static_cast<cudaStream_t>(stream));
+}
+
+int headcast_set_labels(headcast_ctx* c, const int32_t* labels) {
+  if (!c || !labels) return HC_ERR_INVALID_ARG;
+  if (c->state != STATE_FILLING) return fail(c, HC_ERR_STATE, "labels are fixed once the cache is split");
+  for (int h = 0; h < c->H; ++h)
+    if (labels[h] < 0 || labels[h] > 3) return fail(c, HC_ERR_INVALID_ARG, "label %d of head %d is not an archetype", labels[h], h);
+  c->labels.assign(labels, labels + c->H);
+  c->have_labels = true;
+  return HC_OK;
+}
+
+int headcast_get_labels(const headcast_ctx* c, int32_t* labels) {
+  if (!c || !labels) return HC_ERR_INVALID_ARG;
+  if (!c->have_labels) return HC_ERR_STATE;
+  std::copy(c->labels.begin(), c->labels.end(), labels);
+  return HC_OK;
+}
+
+int headcast_classify(headcast_ctx* c, const void* q, int32_t* labels_host, float* scores_host, void* stream) {
+  if (!c || !labels_host) return HC_ERR_INVALID_ARG;
+  if (!aligned16(q)) return fail(c, HC_ERR_INVALID_ARG, "q must be a 16-byte aligned device pointer");
+  if (c->state != STATE_FILLING) return fail(c, HC_ERR_STATE, "classification runs on the monolithic cache, before the split");
+  if (n_filled(c) < 2) return fail(c, HC_ERR_STATE, "classification needs at least two cached blocks");
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t rows = static_cast<size_t>(c->L) * c->H;
+  HC_CUDA(c, c->cls_o.reserve(4 * rows * c->D));
+  HC_CUDA(c, c->cls_lse.reserve(5 * rows));
+  HC_CUDA(c, c->cls_tok.reserve(TOK_N * rows));
+  HC_CUDA(c, c->cls_scores.reserve(static_cast<size_t>(c->H) * HC_N_SCORES));
+  HC_CUDA(c, c->cls_labels.reserve(c->H));
+  const int newest = c->slots.back();
+  {  // reference (Eq. 2), Sink proxy and Dummy proxy share one launch
+    std::vector<Proto> protos;
+    for (int h = 0; h < c->H; ++h) {
+      WorkItem w = range_item(h, MAP_MONO, h * c->D, 0, n_filled(c) * c->L);
+      w.out_mode = OUT_F32_LSE;
+      w.out_slot = 0;
+      add_query_pairs(protos, w, c->L, w.tiles_per_seg);
+      w = range_item(h, MAP_MONO, h * c->D, 0, c->L);
+      w.out_mode = OUT_F32_LSE;
+      w.out_slot = 1;
+      add_query_pairs(protos, w, c->L, w.tiles_per_seg);
+      w = range_item(h, MAP_MONO, h * c->D, static_cast<long long>(newest) * c->L, c->L);
+      w.out_mode = OUT_F32_LSE;
+      w.out_slot = 2;
+      add_query_pairs(protos, w, c->L, w.tiles_per_seg);
+    }
+    finalize_schedule(c, c->sched_cls, protos, false);
+  }
+  {  // Spatial proxy: per query-tile pair, the band of grid rows within r of any of its queries, in every cached frame
+    std::vector<Proto> protos;
+    const int r = c->cfg.proxy_radius;
+    for (int h = 0; h < c->H; ++h)
+      for (int q0 = 0; q0 < c->L; q0 += 256) {
+        const int q1 = std::min(c->L, q0 + 256) - 1;
+        int a = 0, b = c->T_f;
+        if (q0 / c->T_f == q1 / c->T_f) {
+          const int ylo = std::max(0, (q0 % c->T_f) / c->G_w - r), yhi = std::min(c->G_h - 1, (q1 % c->T_f) / c->G_w + r);
+          a = ylo * c->G_w;
+          b = (yhi + 1) * c->G_w;
+        }
+        WorkItem w = range_item(h, MAP_MONO, h * c->D, a, b - a);
+        w.seg_stride = c->T_f;
+        w.out_mode = OUT_F32_LSE;
+        w.out_slot = 3;
+        Proto p;
+        p.w = w;
+        p.w.q_start[0] = q0;
+        p.w.q_start[1] = q0 + 128;
+        p.w.q_count[0] = std::min(128, c->L - q0);
+        p.w.q_count[1] = std::max(0, std::min(128, c->L - q0 - 128));
+        p.n_tiles = w.tiles_per_seg * n_filled(c) * c->F_b;
+        p.w.tile_begin = 0;
+        p.w.tile_end = p.n_tiles;
+        protos.push_back(p);
+      }
+    finalize_schedule(c, c->sched_proxy, protos, false);
+  }
+  int rc = run_schedule(c, c->sched_cls, q, nullptr, false, st);
+  if (rc != HC_OK) return rc;
+  rc = run_schedule(c, c->sched_proxy, q, nullptr, true, st);
+  if (rc != HC_OK) return rc;
+  {
+    const long long warps = static_cast<long long>(rows);
+    const unsigned blocks = static_cast<unsigned>((warps * 32 + 255) / 256);
+    if (c->D == 128)
+      token_scores_kernel<128><<<blocks, 256, 0, st>>>(c->cls_o.ptr, c->cls_lse.ptr, c->cls_tok.ptr, c->L, c->H);
+    else
+      token_scores_kernel<64><<<blocks, 256, 0, st>>>(c->cls_o.ptr, c->cls_lse.ptr, c->cls_tok.ptr, c->L, c->H);
+    HC_CUDA(c, cudaGetLastError());
+    ++c->launches;
+    DecideParams d;
+    d.tok = c->cls_tok.ptr;
+    d.scores = c->cls_scores.ptr;
+    d.labels = c->cls_labels.ptr;
+    d.L = c->L;
+    d.H = c->H;
+    d.D = c->D;
+    const double rank = 0.05 * (c->L - 1);
+    d.rank_lo = static_cast<int32_t>(std::floor(rank));
+    d.rank_frac = static_cast<float>(rank - std::floor(rank));
+    d.theta_sink = c->cfg.theta_sink;
+    d.theta_dummy = c->cfg.theta_dummy;
+    d.theta_spatial = c->cfg.theta_spatial;
+    d.theta_score = c->cfg.theta_score;
+    d.gamma = c->cfg.gamma;
+    head_decide_kernel<<<c->H, 512, 0, st>>>(d);
+    HC_CUDA(c, cudaGetLastError());
+    ++c->launches;
+  }
+  std::vector<float> scores(static_cast<size_t>(c->H) * HC_N_SCORES);
+  HC_CUDA(c, cudaMemcpyAsync(labels_host, c->cls_labels.ptr, c->H * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+  HC_CUDA(c, cudaMemcpyAsync(scores.data(), c->cls_scores.ptr, scores.size() * sizeof(float), cudaMemcpyDeviceToHost, st));
+  rc = read_status(c, st);
+  if (rc != HC_OK) return rc;
+  if (scores_host) std::copy(scores.begin(), scores.end(), scores_host);
+  c->labels.assign(labels_host, labels_host + c->H);
+  c->have_labels = true;
+  return HC_OK;
+}
+
+int headcast_split_cache(headcast_ctx* c, void* stream) {
+  if (!c) return HC_ERR_INVALID_ARG;
+  if (c->state != STATE_FILLING) return fail(c, HC_ERR_STATE, "the cache is already split");
+  if (!c->have_labels) return fail(c, HC_ERR_STATE, "no labels: call headcast_classify or headcast_set_labels first");
+  if (c->slots.empty()) return fail(c, HC_ERR_STATE, "the cache is empty");
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  assign_classes(c);
+  const size_t esz = sizeof(__nv_bfloat16);
+  const int n_sd = c->n_cls[CLS_SINK] + c->n_cls[CLS_DUMMY];
+  const size_t sd_bytes = static_cast<size_t>(n_sd) * c->L * c->D * esz;
+  const size_t g_bytes = cache_elems(c, c->n_cls[CLS_GLOBAL]) * esz;
+  const size_t sp_bytes = cache_elems(c, c->n_cls[CLS_SPATIAL]) * esz;
+  struct { __nv_bfloat16** p; size_t bytes; } bufs[] = {{&c->sd_k, sd_bytes}, {&c->sd_v, sd_bytes}, {&c->g_k, g_bytes},
+                                                        {&c->g_v, g_bytes},   {&c->sp_k, sp_bytes}, {&c->sp_v, sp_bytes}};
+  for (auto& b : bufs) {
+    if (b.bytes == 0) continue;
+    cudaError_t e = cudaMalloc(b.p, b.bytes);
+    if (e == cudaSuccess) e = cudaMemsetAsync(*b.p, 0, b.bytes, st);
+    if (e != cudaSuccess) {
+      for (auto& f : bufs)
+        if (*f.p) { cudaFree(*f.p); *f.p = nullptr; }
+      return fail(c, e == cudaErrorMemoryAllocation ? HC_ERR_NOMEM : HC_ERR_CUDA, "allocating the per-archetype buffers: %s",
+                  cudaGetErrorString(e));
+    }
+  }
+  const size_t block_elems = static_cast<size_t>(c->L) * c->H * c->D;
+  for (size_t i = 0; i < c->slots.size(); ++i) {
+    RouteParams r;
+    fill_route(c, r);
+    const int slot = c->slots[i];
+    r.src_k = reinterpret_cast<const uint4*>(c->mono_k + slot * block_elems);
+    r.src_v = reinterpret_cast<const uint4*>(c->mono_v + slot * block_elems);
+    r.slot = slot;
+    r.copy_mono = 0;
+    r.copy_sink = (i == 0);
+    r.copy_dummy = (i + 1 == c->slots.size());
+    r.copy_window = 1;
+    int rc = launch_route(c, r, st);
+    if (rc != HC_OK) return rc;
+  }
+  if (!c->cfg.keep_monolithic) {
+    HC_CUDA(c, cudaStreamSynchronize(st));
+    cudaFree(c->mono_k);
+    cudaFree(c->mono_v);
+    c->mono_k = c->mono_v = nullptr;
+  }
+  c->state = STATE_SPLIT;
+  c->sched_hc.key_filled = -1;
+  return build_maps(c);
+}
+
+int headcast_attend(headcast_ctx* c, const void* q, void* out, void* stream) {
+  if (!c) return HC_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(out)) return fail(c, HC_ERR_INVALID_ARG, "q/out must be 16-byte aligned device pointers");
+  if (c->state != STATE_SPLIT) return fail(c, HC_ERR_STATE, "head-specific attention needs the split cache");
+  if (c->sched_hc.key_filled != n_filled(c)) build_headcast_schedule(c, c->sched_hc);
+  return run_schedule(c, c->sched_hc, q, out, false, static_cast<cudaStream_t>(stream));
+}
+
+int headcast_export_cache(headcast_ctx* c, int32_t head, void* k_out, void* v_out, int32_t* n_tokens_host, void* stream) {
+  if (!c || head < 0 || head >= c->H) return HC_ERR_INVALID_ARG;
+  if ((k_out && !aligned16(k_out)) || (v_out && !aligned16(v_out))) return fail(c, HC_ERR_INVALID_ARG, "outputs must be 16-byte aligned");
+  ExportParams e;
+  std::memset(&e, 0, sizeof(e));
+  e.dst_k = static_cast<uint4*>(k_out);
+  e.dst_v = static_cast<uint4*>(v_out);
+  e.sp_base = c->sp_base;
+  e.sp_nc = c->sp_nc;
+  e.L = c->L;
+  e.H = c->H;
+  e.chunks = c->CH;
+  e.tokens_per_frame = c->T_f;
+  e.frames_per_block = c->F_b;
+  e.n_blocks = c->n_blk;
+  const int cl = (c->state == STATE_SPLIT) ? c->cls[head] : CLS_NONE;
+  if (cl == CLS_NONE) {
+    e.layout = 0; e.head = head; e.src_k = reinterpret_cast<const uint4*>(c->mono_k); e.src_v = reinterpret_cast<const uint4*>(c->mono_v);
+  } else if (cl == CLS_GLOBAL) {
+    e.layout = 1; e.head = c->idx[head]; e.src_k = reinterpret_cast<const uint4*>(c->g_k); e.src_v = reinterpret_cast<const uint4*>(c->g_v);
+  } else if (cl == CLS_SPATIAL) {
+    e.layout = 2; e.head = c->idx[head]; e.src_k = reinterpret_cast<const uint4*>(c->sp_k); e.src_v = reinterpret_cast<const uint4*>(c->sp_v);
+  } else {
+    e.layout = 3; e.head = (cl == CLS_SINK) ? c->idx[head] : c->n_cls[CLS_SINK] + c->idx[head];
+    e.src_k = reinterpret_cast<const uint4*>(c->sd_k); e.src_v = reinterpret_cast<const uint4*>(c->sd_v);
+  }
+  if (e.layout == 3) {
+    e.n_logical = c->slots.empty() ? 0 : 1;
+    e.slots[0] = 0;
+  } else {
+    e.n_logical = n_filled(c);
+    for (int i = 0; i < e.n_logical; ++i) e.slots[i] = c->slots[i];
+  }
+  if (n_tokens_host) *n_tokens_host = e.n_logical * c->L;
+  if (e.n_logical == 0 || (!k_out && !v_out)) return HC_OK;
+  const long long total = static_cast<long long>(e.n_logical) * c->L * c->CH;
+  const int blocks = static_cast<int>(std::min<long long>((total + 255) / 256, c->n_sm * 16LL));
+  export_head_kernel<<<blocks, 256, 0, static_cast<cudaStream_t>(stream)>>>(e);
+  HC_CUDA(c, cudaGetLastError());
+  ++c->launches;
+  return HC_OK;
+}
+
+int headcast_n_filled(const headcast_ctx* c) { return c ? n_filled(c) : HC_ERR_INVALID_ARG; }
+
+int64_t headcast_launch_count(const headcast_ctx* c) { return c ? c->launches : 0; }
+
+double headcast_attend_flops(const headcast_ctx* c, int32_t dense) {
+  if (!c) return 0.0;
+  const int nf = n_filled(c);
+  if (dense) return 4.0 * c->H * static_cast<double>(c->L) * nf * c->L * c->D;
+  if (!c->have_labels) return 0.0;
+  double cell_sq = 0.0;
+  for (const CellGeom& g : c->cells) cell_sq += static_cast<double>(g.ch * g.cw) * (g.ch * g.cw);
+  double f = 0.0;
+  for (int h = 0; h < c->H; ++h) {
+    if (c->labels[h] == HC_SINK || c->labels[h] == HC_DUMMY) f += 4.0 * c->L * static_cast<double>(c->L) * c->D;
+    else if (c->labels[h] == HC_GLOBAL) f += 4.0 * c->L * static_cast<double>(nf) * c->L * c->D;
+    else f += 4.0 * c->F_b * static_cast<double>(nf) * c->F_b * cell_sq * c->D;
+  }
+  return f;
+}
+
+int headcast_check(headcast_ctx* c, void* stream) {
+  if (!c) return HC_ERR_INVALID_ARG;
+  return read_status(c, static_cast<cudaStream_t>(stream));
+}
+
+const char* headcast_last_error(const headcast_ctx* c) { return c ? c->err.c_str() : "null context"; }
+
+}  // extern "C"

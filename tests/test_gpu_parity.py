@@ -1,0 +1,236 @@
+"""GPU parity: the CUDA library (through its C ABI) against the float64 CPU oracle on the same seeded bytes.
+
+Bars: cache contents and labels bit-exact; attention outputs (bf16 Q/K/V, fp32 accumulation, bf16 output)
+within max-abs 2e-2 and mean-abs 2e-3 of the oracle; classification scores within 5e-3 (cosines, masses)
+and 1e-2 (score).
+"""
+import numpy as np
+import pytest
+
+from oracle import headcast_oracle as orc
+from paper_2607_20125_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+MAX_ABS, MEAN_ABS = 2e-2, 2e-3
+
+
+def to_dev(bits):
+    import torch
+    return torch.from_numpy(bits.view(np.int16)).view(torch.bfloat16).cuda()
+
+
+def to_f64(t):
+    import torch
+    return t.float().cpu().numpy().astype(np.float64)
+
+
+def geometry(w, **kw):
+    return orc.Geometry.make(w.grid_h, w.grid_w, w.frames_per_block, w.cell_h, w.cell_w, **kw)
+
+
+class Pair:
+    """The library context and the oracle's cache model, fed the same blocks."""
+
+    def __init__(self, w, keep_monolithic=True, **kw):
+        from paper_2607_20125_b200.binding import HeadCast
+        self.w = w
+        self.hc = HeadCast.from_workload(w, keep_monolithic=keep_monolithic, **kw)
+        self.cache = orc.CacheModel(w.n_blocks, w.n_heads)
+        self.geom = geometry(w, row_edges=kw.get("row_edges"), col_edges=kw.get("col_edges"))
+        self.next_block = 0
+
+    def append(self, n=1):
+        for _ in range(n):
+            k, v = synth.make_kv(self.w, self.next_block)
+            self.hc.append(to_dev(k), to_dev(v))
+            self.cache.append(k, v)
+            self.next_block += 1
+
+    def check_cache(self):
+        for h in range(self.w.n_heads):
+            k, v = self.hc.export_cache(h)
+            ko, vo = self.cache.head_kv_bits(h)
+            assert k.shape == ko.shape, (h, k.shape, ko.shape)
+            assert np.array_equal(k, ko) and np.array_equal(v, vo), f"cache of head {h} differs"
+
+    def check_attention(self, dense, rows=None, step=0):
+        import torch
+        q = synth.make_q(self.w, self.next_block - 1, step)
+        out = torch.full((self.w.block_tokens, self.w.n_heads, self.w.head_dim), float("nan"),
+                         dtype=torch.bfloat16, device="cuda")
+        (self.hc.full_attend if dense else self.hc.attend)(to_dev(q), out)
+        self.hc.check()
+        got = to_f64(out)
+        assert np.isfinite(got).all(), "rows were left unwritten or are not finite"
+        if dense:
+            want, _ = orc.full_attend(q, self.cache, rows=rows)
+        else:
+            want = orc.attend(q, self.cache, self.geom, rows=rows)
+        if rows is not None:
+            got = got[rows]
+        err = np.abs(got - want)
+        per_head = err.mean(axis=(0, 2))
+        assert err.max() <= MAX_ABS, (err.max(), np.unravel_index(err.argmax(), err.shape))
+        assert per_head.max() <= MEAN_ABS, per_head
+        return err
+
+
+def run_pipeline(w, fill, extra, labels=None, rows=None, **kw):
+    p = Pair(w, **kw)
+    p.append(fill)
+    p.check_cache()
+    p.check_attention(dense=True, rows=rows)
+    p.hc.set_labels(w.labels if labels is None else labels)
+    p.hc.split_cache()
+    p.cache.split(w.labels if labels is None else labels)
+    p.check_cache()
+    p.check_attention(dense=False, rows=rows)
+    for i in range(extra):
+        p.append()
+        p.check_cache()
+        p.check_attention(dense=False, rows=rows, step=i % 4)
+    p.check_attention(dense=True, rows=rows)
+    return p
+
+
+@pytest.mark.parametrize("cell", [10, 4])
+def test_tiny_all_rows(cell):
+    w = synth.tiny(cell=cell)
+    run_pipeline(w, fill=5, extra=3)
+
+
+def test_small_ragged_split_during_growth_then_roll():
+    # 13x22 grid, d=128: L = 858 (6.7 query tiles), cells of 5..7 x 7..8 tokens, window of 4 blocks;
+    # split with 2 of 4 blocks cached, then grow to full and roll three times
+    w = synth.small()
+    run_pipeline(w, fill=2, extra=5)
+
+
+def test_single_block_cache_and_first_block_is_newest():
+    w = synth.small(n_blocks=3)
+    p = Pair(w)
+    p.append(1)
+    p.check_attention(dense=True)
+    p.hc.set_labels(w.labels)
+    p.hc.split_cache()
+    p.cache.split(w.labels)
+    p.check_cache()
+    p.check_attention(dense=False)
+
+
+@pytest.mark.parametrize("labels", [[orc.GLOBAL] * 6, [orc.SPATIAL] * 6, [orc.SINK, orc.DUMMY] * 3])
+def test_archetype_groups_may_be_empty(labels):
+    w = synth.small(n_blocks=3)
+    run_pipeline(w, fill=3, extra=1, labels=labels)
+
+
+def test_explicit_cell_edges_one_row_cells():
+    w = synth.small(n_blocks=3)
+    rows_e = [0, 1, 2, 7, 13]
+    cols_e = [0, 21, 22]
+    run_pipeline(w, fill=3, extra=1, row_edges=rows_e, col_edges=cols_e)
+
+
+def test_zero_queries_give_the_mean_value_of_each_key_set():
+    import torch
+    w = synth.small(n_blocks=3)
+    p = Pair(w)
+    p.append(3)
+    p.hc.set_labels(w.labels)
+    p.hc.split_cache()
+    p.cache.split(w.labels)
+    q = torch.zeros((w.block_tokens, w.n_heads, w.head_dim), dtype=torch.bfloat16, device="cuda")
+    out = torch.empty_like(q)
+    p.hc.attend(q, out)
+    p.hc.check()
+    got = to_f64(out)
+    L = w.block_tokens
+    for h, lab in enumerate(w.labels):
+        v = orc.widen_bf16(p.cache.mono_kv_bits(h)[1])
+        if lab == orc.SINK:
+            assert np.abs(got[:, h] - v[:L].mean(axis=0)).max() < 2e-3
+        elif lab == orc.DUMMY:
+            assert np.abs(got[:, h] - v[-L:].mean(axis=0)).max() < 2e-3
+        elif lab == orc.GLOBAL:
+            assert np.abs(got[:, h] - v.mean(axis=0)).max() < 2e-3
+        else:
+            cells = p.geom.cell_of(np.arange(v.shape[0]))
+            for t in (0, 21, 300, L - 1):
+                want = v[cells == p.geom.cell_of(np.array([t]))[0]].mean(axis=0)
+                assert np.abs(got[t, h] - want).max() < 4e-3
+
+
+def test_wrong_state_calls_change_nothing():
+    import torch
+    from paper_2607_20125_b200.binding import HeadCastError
+    w = synth.tiny()
+    p = Pair(w, keep_monolithic=False)
+    q = to_dev(synth.make_q(w, 0, 0))
+    out = torch.empty_like(q)
+    for call in (lambda: p.hc.full_attend(q, out), lambda: p.hc.attend(q, out), lambda: p.hc.split_cache(),
+                 lambda: p.hc.classify(q)):
+        with pytest.raises(HeadCastError) as e:
+            call()
+        assert e.value.code == -2
+    p.append(1)
+    with pytest.raises(HeadCastError) as e:
+        p.hc.classify(q)  # one cached block: first block == newest block
+    assert e.value.code == -2
+    with pytest.raises(HeadCastError) as e:
+        p.hc.set_labels([0, 1, 2, 7])
+    assert e.value.code == -1
+    p.append(1)
+    p.hc.set_labels(w.labels)
+    p.hc.split_cache()
+    p.cache.split(w.labels)
+    with pytest.raises(HeadCastError) as e:
+        p.hc.full_attend(q, out)  # monolithic cache was released
+    assert e.value.code == -2
+    with pytest.raises(HeadCastError):
+        p.hc.set_labels(w.labels)
+    with pytest.raises(HeadCastError) as e:
+        p.hc.attend(q[1:].reshape(-1)[1:], out)  # misaligned pointer
+    assert e.value.code == -1
+    p.check_cache()
+    assert p.hc.n_filled() == 2
+
+
+def check_classify(w, fill, rows=None):
+    p = Pair(w)
+    p.append(fill)
+    q = synth.make_q(w, fill - 1, 0)
+    labels, scores = p.hc.classify(to_dev(q))
+    want_labels, want = orc.classify(q, p.cache, p.geom, rows=rows)
+    assert tuple(labels) == tuple(want_labels) == tuple(w.labels)
+    if rows is None:
+        d = np.abs(scores.astype(np.float64) - want)
+        assert d[:, [0, 1, 2, 6, 7, 8, 9]].max() <= 5e-3, d
+        assert d[:, [3, 5]].max() <= 1e-2 and d[:, 4].max() <= 2e-3, d
+    assert p.hc.get_labels() == list(w.labels)
+    return p
+
+
+@pytest.mark.parametrize("cell", [10, 4])
+def test_classify_tiny(cell):
+    p = check_classify(synth.tiny(cell=cell), 5)
+    p.hc.split_cache()
+    p.cache.split(p.w.labels)
+    p.check_cache()
+    p.check_attention(dense=False)
+
+
+def test_classify_small_with_ring_rolled_before_classification():
+    # 6 appends into a 4-block cache: the newest block is not the last physical slot
+    check_classify(synth.small(), 6)
+
+
+def test_classify_small_two_blocks_no_middle():
+    check_classify(synth.small(), 2)
+
+
+def test_480p_sampled_rows():
+    w = synth.wan("480p")
+    rows = synth.sample_rows(w, n_random=128)
+    p = run_pipeline(w, fill=7, extra=1, rows=rows)
+    assert abs(p.hc.attend_flops(False) / 1e9 - 312.5) < 0.5 and abs(p.hc.attend_flops(True) / 1e9 - 942.0) < 0.5
