@@ -1,0 +1,384 @@
+#!/usr/bin/env python
+"""Benchmark of the HeadCast attention path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload 480p|720p|1080p|tiny] [--impl reference]
+
+A *step* is one block-denoise-step of the steady state: one ``headcast_attend`` call, preceded every 4th step by
+the per-block ``headcast_append`` (4 denoise steps reuse the cache).  The one-time phases of the path (warm-up
+appends, dense attention, classification, split) are timed once and reported in ``phases``.  Rank 0 prints ONE
+JSON line.  ``--impl reference`` times the float64 CPU oracle on a bounded sample instead.
+
+The path does not shard (one attention layer on one GPU): with ``--gpus N`` every rank runs an independent
+replica and the slowest rank's time is reported.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2607_20125_b200 import synth  # noqa: E402
+
+METRIC = "headcast_attn_ms_per_block_step"
+STEPS_PER_BLOCK = 4
+# dram__bytes_read.sum + dram__bytes_write.sum of one attention-kernel launch, from the ncu captures summarised
+# under profiles/ (None where not captured at that size)
+NCU_TRAFFIC_BYTES = {"480p": None, "720p": None, "1080p": None, "tiny": None}
+
+
+def workload_of(name: str):
+    return synth.tiny() if name == "tiny" else synth.wan(name)
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return {"tflops": d["bf16_tflops"], "tflops_sustained": d.get("bf16_tflops_sustained"), "hbm_gbs": d["hbm_gbs"],
+                "source": "measured"}
+    return {"tflops": 1590.0, "tflops_sustained": 1400.0, "hbm_gbs": 6650.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the timed region runs (read-only)."""
+
+    def __init__(self, index: int):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.handle = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.handle, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _run(self):
+        nv = self.nv
+        names = {"hw_slowdown": "nvmlClocksEventReasonHwSlowdown", "hw_thermal_slowdown": "nvmlClocksEventReasonHwThermalSlowdown",
+                 "sw_thermal_slowdown": "nvmlClocksEventReasonSwThermalSlowdown", "sw_power_cap": "nvmlClocksEventReasonSwPowerCap"}
+        bits = {k: getattr(nv, v, None) or getattr(nv, v.replace("Event", "Throttle"), 0) for k, v in names.items()}
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.handle, nv.NVML_CLOCK_SM))
+                try:
+                    r = nv.nvmlDeviceGetCurrentClocksEventReasons(self.handle)
+                except Exception:
+                    r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.handle)
+                self.reasons.update(k for k, b in bits.items() if b and (r & b))
+            except Exception:
+                pass
+            time.sleep(0.004)
+
+    def __enter__(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0}
+        return {"sm_mhz": float(np.median(self.samples)), "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+def to_dev(bits, torch):
+    return torch.from_numpy(bits.view(np.int16)).view(torch.bfloat16).cuda()
+
+
+def timed(torch, fn, flush, reps):
+    """Mean CUDA-event time of fn() over reps calls, L2 flushed (outside the events) before each."""
+    total = 0.0
+    for _ in range(reps):
+        flush()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        fn()
+        b.record()
+        b.synchronize()
+        total += a.elapsed_time(b)
+    return total / reps
+
+
+_ORACLE_STATE = {}
+
+
+def _oracle_state(w):
+    """Cache model, geometry, queries and sampled rows of the oracle arm (built once per process)."""
+    if w.name not in _ORACLE_STATE:
+        from oracle import headcast_oracle as orc
+        geom = orc.Geometry.make(w.grid_h, w.grid_w, w.frames_per_block, w.cell_h, w.cell_w)
+        cache = orc.CacheModel(w.n_blocks, w.n_heads)
+        for b in range(w.n_blocks):
+            cache.append(*synth.make_kv(w, b))
+        cache.split(w.labels)
+        q = synth.make_q(w, w.n_blocks - 1, 0)
+        rows = synth.sample_rows(w, n_random=64)
+        t0 = time.perf_counter()
+        orc.attend(q, cache, geom, rows=rows[:32])
+        per_row = (time.perf_counter() - t0) / 32
+        _ORACLE_STATE[w.name] = (orc, geom, cache, q, rows, per_row)
+    return _ORACLE_STATE[w.name]
+
+
+def cpu_baseline(w, target_s=12.0):
+    """The oracle, as it stands, on a bounded sample of the same workload: head-specific attention for a few query
+    rows of every head, extrapolated linearly to the whole block (rows are independent)."""
+    orc, geom, cache, q, rows, per_row = _oracle_state(w)
+    n = int(max(32, min(rows.size, target_s / max(per_row, 1e-9))))
+    t0 = time.perf_counter()
+    orc.attend(q, cache, geom, rows=rows[:n])
+    dt = time.perf_counter() - t0
+    try:
+        from threadpoolctl import threadpool_info
+        cores = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        cores = os.cpu_count()
+    return {"value": dt / n * w.block_tokens * 1e3, "unit": "ms", "cores": int(cores), "kind": "oracle",
+            "sample": f"{n} of {w.block_tokens} query rows of every head, one attend; {dt:.1f} s measured, extrapolated linearly"}
+
+
+def run_reference(args, w):
+    """--impl reference: the CPU oracle as the reference arm (bounded sample per step)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    per_step = []
+    base = None
+    for i in range(args.warmup + args.steps):
+        base = cpu_baseline(w, target_s=max(2.0, min(12.0, 150.0 / (args.warmup + args.steps))))
+        if i >= args.warmup:
+            per_step.append(base["value"])
+    value = float(np.mean(per_step))
+    base["value"] = value
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": "ms", "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": value, "higher_is_better": False, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": w.name, "heads": w.n_heads, "head_dim": w.head_dim, "grid": [w.grid_h, w.grid_w],
+                       "block_tokens": w.block_tokens, "kv_tokens": w.n_blocks * w.block_tokens},
+            "cpu_baseline": base, "e2e": {"value": value, "unit": "ms", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=8)
+    ap.add_argument("--workload", default="480p", choices=["tiny", "480p", "720p", "1080p"])
+    ap.add_argument("--impl", default="headcast", choices=["headcast", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-phases", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+    w = workload_of(args.workload)
+    if args.impl == "reference":
+        return run_reference(args, w)
+
+    import torch
+    from paper_2607_20125_b200.binding import HeadCast
+
+    rank, world = int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    peaks = measured_peaks()
+
+    L, H, D = w.block_tokens, w.n_heads, w.head_dim
+    flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    flush = lambda: flush_buf.zero_()
+
+    hc = HeadCast.from_workload(w, keep_monolithic=True)
+    n_extra = 3  # generated blocks fed round-robin once the cache rolls, each with its own 4 denoise-step queries
+    kv = [tuple(to_dev(t, torch) for t in synth.make_kv(w, b)) for b in range(w.n_blocks + n_extra)]
+    q_fill = to_dev(synth.make_q(w, w.n_blocks - 1, 0), torch)
+    q_extra = [[to_dev(synth.make_q(w, w.n_blocks + e, s), torch) for s in range(STEPS_PER_BLOCK)] for e in range(n_extra)]
+    qs = [q_fill]
+    out = torch.empty_like(q_fill)
+    phases = {}
+
+    # ---- one-time phases: warm-up appends, dense attention, classification, split
+    for b in range(w.n_blocks):
+        hc.append(*kv[b])
+    torch.cuda.synchronize()
+    block_bytes = 2 * L * H * D * 2
+    if not args.no_phases:
+        hc.set_kernel_timing(True)
+        for _ in range(3):
+            hc.full_attend(qs[0], out)
+        dense_ms = timed(torch, lambda: hc.full_attend(qs[0], out), flush, 10)
+        phases["dense_full_attend_ms"] = dense_ms
+        phases["dense_tflops"] = hc.attend_flops(True) / dense_ms / 1e9
+        t0 = time.perf_counter()
+        labels, scores = hc.classify(qs[0])
+        torch.cuda.synchronize()
+        t_first = (time.perf_counter() - t0) * 1e3
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        flush()
+        a.record()
+        labels, scores = hc.classify(qs[0])
+        b.record()
+        b.synchronize()
+        phases["classify_ms"] = a.elapsed_time(b)
+        phases["classify_first_call_ms"] = t_first
+        phases["labels_match_planted"] = bool(tuple(int(v) for v in labels) == tuple(w.labels))
+        t = timed(torch, lambda: hc.append(*kv[w.n_blocks]), flush, 5)  # monolithic ring append (rolls)
+        phases["append_monolithic_ms"] = t
+        phases["append_monolithic_gbs"] = 2 * block_bytes / t / 1e6
+    else:
+        hc.set_labels(w.labels)
+        hc.set_kernel_timing(True)
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    flush()
+    a.record()
+    hc.split_cache()
+    b.record()
+    b.synchronize()
+    n_sd = sum(1 for v in w.labels if v in (synth.SINK, synth.DUMMY))
+    kept_bytes = 2 * 2 * L * D * (n_sd + (H - n_sd) * w.n_blocks)
+    phases["split_ms"] = a.elapsed_time(b)  # includes the allocation of the per-archetype buffers
+    phases["split_gbs"] = 2 * kept_bytes / phases["split_ms"] / 1e6
+
+    n_sink = sum(1 for v in w.labels if v == synth.SINK)
+    append_bytes = block_bytes + 2 * L * (H - n_sink) * D * 2 + block_bytes  # read + per-archetype writes + monolithic copy
+
+    state = {"i": 0}
+
+    def step():
+        i = state["i"]
+        e = (i // STEPS_PER_BLOCK) % n_extra
+        if i % STEPS_PER_BLOCK == 0:
+            hc.append(*kv[w.n_blocks + e])
+        hc.attend(q_extra[e][i % STEPS_PER_BLOCK], out)
+        state["i"] = i + 1
+
+    for _ in range(args.warmup):
+        step()
+    hc.check()
+    state["i"] = 0
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    launches0 = hc.launch_count()
+    step_ms, kernel_ms, append_ms = [], [], []
+    with ClockSampler(local) as clocks:
+        for i in range(args.steps):
+            flush()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            m = torch.cuda.Event(enable_timing=True)
+            a.record()
+            e = (i // STEPS_PER_BLOCK) % n_extra
+            if i % STEPS_PER_BLOCK == 0:
+                hc.append(*kv[w.n_blocks + e])
+                m.record()
+            hc.attend(q_extra[e][i % STEPS_PER_BLOCK], out)
+            b.record()
+            b.synchronize()
+            step_ms.append(a.elapsed_time(b))
+            if i % STEPS_PER_BLOCK == 0:
+                append_ms.append(a.elapsed_time(m))
+            kernel_ms.append(hc.last_attention_kernel_ms())
+        torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    hc.check()
+    launches = hc.launch_count() - launches0
+    total_ms = float(np.sum(step_ms))
+    if dist is not None:
+        tt = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        total_ms = float(tt.item())
+    ms_per_step = total_ms / args.steps
+    attend_ms = float(np.mean([s - (append_ms[i // STEPS_PER_BLOCK] if i % STEPS_PER_BLOCK == 0 else 0.0)
+                               for i, s in enumerate(step_ms)]))
+    kern = float(np.mean(kernel_ms))
+    flops = hc.attend_flops(False)
+    phases["append_split_ms"] = float(np.mean(append_ms))
+    phases["append_split_gbs"] = append_bytes / phases["append_split_ms"] / 1e6
+    phases["attend_ms"] = attend_ms
+    phases["attend_tflops"] = flops / attend_ms / 1e9
+    if "dense_full_attend_ms" in phases:
+        phases["speedup_vs_dense"] = phases["dense_full_attend_ms"] / attend_ms
+        phases["ideal_speedup_by_flops"] = hc.attend_flops(True) / flops
+
+    # ---- end to end through the same calls with host buffers (pinned), copies inside the timed region
+    host_q = [q.cpu().pin_memory() for q in q_extra[0]]
+    host_kv = [(k.cpu().pin_memory(), v.cpu().pin_memory()) for k, v in kv[w.n_blocks:w.n_blocks + 2]]
+    host_out = torch.empty_like(host_q[0]).pin_memory()
+    dq, dk, dv = torch.empty_like(q_fill), torch.empty_like(kv[0][0]), torch.empty_like(kv[0][1])
+    e2e_steps = min(args.steps, 40)
+    e2e_ms = []
+    for i in range(-3, e2e_steps):
+        flush()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        if i % STEPS_PER_BLOCK == 0:
+            dk.copy_(host_kv[(i // STEPS_PER_BLOCK) % 2][0], non_blocking=True)
+            dv.copy_(host_kv[(i // STEPS_PER_BLOCK) % 2][1], non_blocking=True)
+            hc.append(dk, dv)
+        dq.copy_(host_q[i % STEPS_PER_BLOCK], non_blocking=True)
+        hc.attend(dq, out)
+        host_out.copy_(out, non_blocking=True)
+        b.record()
+        b.synchronize()
+        if i >= 0:
+            e2e_ms.append(a.elapsed_time(b))
+    e2e = float(np.sum(e2e_ms)) / e2e_steps
+    if dist is not None:
+        tt = torch.tensor([e2e], device="cuda", dtype=torch.float64)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        e2e = float(tt.item())
+    q_bytes = L * H * D * 2
+
+    if rank != 0:
+        return
+    achieved = flops / kern / 1e9
+    line = {
+        "metric": METRIC, "value": ms_per_step, "unit": "ms", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": w.name, "heads": H, "head_dim": D, "grid": [w.grid_h, w.grid_w], "block_tokens": L,
+                   "kv_tokens": w.n_blocks * L, "head_mix_sink_dummy_spatial_global": [int(sum(1 for v in w.labels if v == c)) for c in range(4)],
+                   "step": "1 attend per step + 1 append per 4 steps", "l2": "flushed between steps (256 MiB memset outside the events)",
+                   "parallelism": "replicas only" if world > 1 else "single GPU"},
+        "clocks": clocks.summary(),
+        "e2e": {"value": e2e, "unit": "ms", "h2d_bytes_per_step": q_bytes + block_bytes // STEPS_PER_BLOCK, "d2h_bytes_per_step": q_bytes},
+        "gpu_launches": int(launches),
+        "roofline": {"bound": "tensor", "kernel": "attn_kernel (tcgen05)", "achieved": achieved, "peak": peaks["tflops"],
+                     "unit": "TFLOP/s", "frac": achieved / peaks["tflops"], "peak_source": peaks["source"] + " (burst bf16 GEMM)",
+                     "frac_of_sustained": achieved / peaks["tflops_sustained"] if peaks["tflops_sustained"] else None,
+                     "frac_of_nominal_2250": achieved / 2250.0, "kernel_ms": kern, "flops_per_launch": flops,
+                     "traffic": NCU_TRAFFIC_BYTES.get(w.name)},
+        "phases": phases,
+        "hbm_peak_gbs": peaks["hbm_gbs"],
+    }
+    if not args.no_cpu_baseline:
+        line["cpu_baseline"] = cpu_baseline(w)
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -147,6 +147,20 @@ int64_t headcast_launch_count(const headcast_ctx* ctx);
  * headcast_full_attend (dense = 1) with the current cache fill and labels. */
 double headcast_attend_flops(const headcast_ctx* ctx, int32_t dense);
 
+/* Benchmark aid.  With enable != 0 every later attention call records CUDA events on its stream directly
+ * before and after its tensor-core attention kernel (not around the small merge kernel that may follow).
+ * headcast_last_attention_kernel_ms waits for the most recent pair and writes the elapsed milliseconds. */
+int headcast_set_kernel_timing(headcast_ctx* ctx, int32_t enable);
+int headcast_last_attention_kernel_ms(headcast_ctx* ctx, float* ms_host);
+
+/* Scheduling aid.  With enable != 0 every later attention launch records, per work item, the GPU global timer
+ * (ns) at which the item's first query tile started and finished.  headcast_read_trace synchronises the device
+ * and writes, for each work item of the most recent attention launch, 8 int64 values to rows_host
+ * ([capacity][8]): CTA index, head, Spatial cell (-1 if none), query rows, key tiles, output mode
+ * (0 final, 1 partial, 2 fp32), start ns, end ns.  *n_items_host receives the item count. */
+int headcast_set_tracing(headcast_ctx* ctx, int32_t enable);
+int headcast_read_trace(headcast_ctx* ctx, int64_t* rows_host, int32_t capacity, int32_t* n_items_host);
+
 /* Synchronises `stream` and reports a device-side status raised by any earlier kernel of this context
  * (HC_ERR_TIMEOUT if a bounded wait expired). */
 int headcast_check(headcast_ctx* ctx, void* stream);

@@ -20,7 +20,9 @@ ERRORS = {0: "HC_OK", -1: "HC_ERR_INVALID_ARG", -2: "HC_ERR_STATE", -3: "HC_ERR_
 EXPORTS = ("headcast_default_config", "headcast_create", "headcast_destroy", "headcast_append",
            "headcast_full_attend", "headcast_classify", "headcast_set_labels", "headcast_get_labels",
            "headcast_split_cache", "headcast_attend", "headcast_export_cache", "headcast_n_filled",
-           "headcast_launch_count", "headcast_attend_flops", "headcast_check", "headcast_last_error")
+           "headcast_launch_count", "headcast_attend_flops", "headcast_check", "headcast_last_error",
+           "headcast_set_kernel_timing", "headcast_last_attention_kernel_ms", "headcast_set_tracing",
+           "headcast_read_trace")
 
 
 class Config(C.Structure):
@@ -67,6 +69,10 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.headcast_attend_flops.argtypes = [vp, C.c_int32]
     lib.headcast_attend_flops.restype = C.c_double
     lib.headcast_check.argtypes = [vp, vp]
+    lib.headcast_set_kernel_timing.argtypes = [vp, C.c_int32]
+    lib.headcast_last_attention_kernel_ms.argtypes = [vp, f32p]
+    lib.headcast_set_tracing.argtypes = [vp, C.c_int32]
+    lib.headcast_read_trace.argtypes = [vp, C.POINTER(C.c_int64), C.c_int32, i32p]
     lib.headcast_last_error.argtypes = [vp]
     lib.headcast_last_error.restype = C.c_char_p
     if path is None:
@@ -188,6 +194,26 @@ class HeadCast:
 
     def attend_flops(self, dense: bool = False) -> float:
         return self.lib.headcast_attend_flops(self._ctx, int(dense))
+
+    def set_kernel_timing(self, enable: bool) -> None:
+        self._check(self.lib.headcast_set_kernel_timing(self._ctx, int(enable)))
+
+    def last_attention_kernel_ms(self) -> float:
+        ms = C.c_float()
+        self._check(self.lib.headcast_last_attention_kernel_ms(self._ctx, C.byref(ms)))
+        return ms.value
+
+    def set_tracing(self, enable: bool) -> None:
+        self._check(self.lib.headcast_set_tracing(self._ctx, int(enable)))
+
+    def read_trace(self):
+        """[n_items, 8] int64: cta, head, cell, query rows, key tiles, output mode, start ns, end ns."""
+        import numpy as np
+        n = C.c_int32()
+        self._check(self.lib.headcast_read_trace(self._ctx, None, 0, C.byref(n)))
+        rows = np.zeros((max(n.value, 1), 8), dtype=np.int64)
+        self._check(self.lib.headcast_read_trace(self._ctx, rows.ctypes.data_as(C.POINTER(C.c_int64)), n.value, C.byref(n)))
+        return rows[: n.value]
 
     def check(self) -> None:
         self._check(self.lib.headcast_check(self._ctx, _stream()))

@@ -7,7 +7,8 @@
 //     product straight from tensor memory);
 //   - K/V tiles (128 keys) arrive through TMA into a 2-stage shared-memory ring (128-byte swizzle);
 //   - two softmax warpgroups, one per query tile, own one query row per thread (online softmax in the
-//     exp2 domain, rescaling of O only when the running maximum grew by more than 2^8);
+//     exp2 domain, two exponentials per special-function operation through packed fp16, rescaling of O
+//     only when the running maximum grew by more than 2^8);
 //   - warp 0 is the TMA producer, warp 1 issues every MMA.
 // Which keys a query tile sees is entirely a property of the work item: a row range of one of the
 // cache buffers (whole window, one block, one Spatial cell) or, for the classification's Spatial
@@ -19,6 +20,17 @@
 #include "tc05.cuh"
 
 namespace hc {
+
+// Development aid (compile with -DHC_TIMELINE): CTA 0 stamps the global timer at the hand-over points of
+// its first key tiles into AttnParams::trace (which must then hold 16 * 64 values beyond the per-item area).
+#ifdef HC_TIMELINE
+#define HC_STAMP(iter, slot)                                                                     \
+  do {                                                                                           \
+    if (p.trace && blockIdx.x == 0 && (iter) < 64) p.trace[p.trace_base + (iter) * 16 + (slot)] = global_timer_ns(); \
+  } while (0)
+#else
+#define HC_STAMP(iter, slot) do { } while (0)
+#endif
 
 struct CellGeom {
   int32_t y0, x0, ch, cw;  // top-left grid position and extent of a deployed Spatial cell
@@ -57,14 +69,22 @@ struct AttnParams {
   int32_t n_heads, tokens_per_frame, grid_w, block_tokens;
   float scale_log2e;       // softmax scale * log2(e)
   int32_t* status;
+  int32_t trace_base;
+  unsigned long long* trace;  // optional [2 * n_items]: globaltimer (ns) when query tile 0's warpgroup starts / ends an item
   // Spatial proxy only
   int32_t radius;
   int32_t mid_seg_lo, mid_seg_hi, last_seg_lo, last_seg_hi;  // segments (cached frames) of the middle / newest blocks
 };
 
-constexpr int ATTN_THREADS = 320;  // warp 0: TMA, warp 1: MMA, warps 2-5 / 6-9: softmax for query tile 0 / 1
+constexpr int ATTN_THREADS = 384;  // warp 0: TMA, warp 1: MMA, warps 2-3 idle, warps 4-7 / 8-11: softmax for query tile 0 / 1
 constexpr int KV_STAGES = 2;
-constexpr float RESCALE_THRESHOLD = 8.0f;  // log2 units
+#ifndef HC_EXP_MODE
+#define HC_EXP_MODE 1
+#endif
+#ifndef HC_RESCALE_THRESHOLD
+#define HC_RESCALE_THRESHOLD 8.0f
+#endif
+constexpr float RESCALE_THRESHOLD = HC_RESCALE_THRESHOLD;  // log2 units
 
 template <int D>
 struct AttnSmem {
@@ -144,11 +164,13 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const AttnParams 
           const int row = w.kv_row0 + seg * w.seg_stride + c * 128;
           const uint32_t st = kt % KV_STAGES, ph = (kt / KV_STAGES) & 1;
           if (!(ok = mbar_wait(&bar_k_free[st], ph ^ 1, abortp, p.status, 11))) break;
+          HC_STAMP(kt, 0);
           mbar_arrive_expect_tx(&bar_k_full[st], SM::TILE_BYTES);
           for (int b = 0; b < NB; ++b)
             tma_load_2d(smem + SM::K_OFF + st * SM::TILE_BYTES + b * SM::BLOCK_BYTES, kmap, w.kv_x0 + 64 * b, row,
                         &bar_k_full[st]);
           if (!(ok = mbar_wait(&bar_v_free[st], ph ^ 1, abortp, p.status, 12))) break;
+          HC_STAMP(kt, 1);
           mbar_arrive_expect_tx(&bar_v_full[st], SM::TILE_BYTES);
           for (int b = 0; b < NB; ++b)
             tma_load_2d(smem + SM::V_OFF + st * SM::TILE_BYTES + b * SM::BLOCK_BYTES, vmap, w.kv_x0 + 64 * b, row,
@@ -174,18 +196,33 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const AttnParams 
                      v_addr = smem_u32(smem + SM::V_OFF);
       uint32_t kt = 0, q_cnt[2] = {0, 0}, p_cnt[2] = {0, 0};
       bool ok = true;
+      // descriptors: the high halves are constant, the low halves are (address >> 4) plus a per-k-step constant
+      const uint32_t kmajor_hi = static_cast<uint32_t>(smem_desc_sw128(0, 16, 1024) >> 32);
+      const uint32_t kmajor_lo = static_cast<uint32_t>(smem_desc_sw128(0, 16, 1024));
+      const uint32_t v_hi = static_cast<uint32_t>(smem_desc_sw128(0, SM::BLOCK_BYTES, 1024) >> 32);
+      const uint32_t v_lo = static_cast<uint32_t>(smem_desc_sw128(0, SM::BLOCK_BYTES, 1024));
       auto issue_qk = [&](int t, uint32_t st) {
+        const uint32_t a0 = kmajor_lo + ((q_addr + t * SM::TILE_BYTES) >> 4);
+        const uint32_t b0 = kmajor_lo + ((k_addr + st * SM::TILE_BYTES) >> 4);
+        const uint32_t d = tmem + S_COL + t * 128;
+#pragma unroll
         for (int kk = 0; kk < QK_STEPS; ++kk) {
-          const uint32_t off = (kk / 4) * SM::BLOCK_BYTES + (kk % 4) * 32;
-          mma_ss(tmem + S_COL + t * 128, smem_desc_sw128(q_addr + t * SM::TILE_BYTES + off, 16, 1024),
-                 smem_desc_sw128(k_addr + st * SM::TILE_BYTES + off, 16, 1024), idesc_s, kk > 0);
+          const uint32_t off = ((kk / 4) * SM::BLOCK_BYTES + (kk % 4) * 32) >> 4;
+          if (kk == 0)
+            mma_ss_lohi<false>(d, a0 + off, kmajor_hi, b0 + off, kmajor_hi, idesc_s);
+          else
+            mma_ss_lohi<true>(d, a0 + off, kmajor_hi, b0 + off, kmajor_hi, idesc_s);
         }
       };
       auto issue_pv = [&](int t, uint32_t st, bool accumulate) {
-        for (int kk = 0; kk < PV_STEPS; ++kk)
-          mma_ts(tmem + O_COL + t * 128, tmem + S_COL + t * 128 + kk * 8,
-                 smem_desc_sw128(v_addr + st * SM::TILE_BYTES + kk * 2048, SM::BLOCK_BYTES, 1024), idesc_o,
-                 (accumulate || kk > 0) ? 1u : 0u);
+        const uint32_t b0 = v_lo + ((v_addr + st * SM::TILE_BYTES) >> 4);
+        const uint32_t d = tmem + O_COL + t * 128, a = tmem + S_COL + t * 128;
+        if (accumulate)
+          mma_ts_lohi<true>(d, a, b0, v_hi, idesc_o);
+        else
+          mma_ts_lohi<false>(d, a, b0, v_hi, idesc_o);
+#pragma unroll
+        for (int kk = 1; kk < PV_STEPS; ++kk) mma_ts_lohi<true>(d, a + kk * 8, b0 + ((kk * 2048) >> 4), v_hi, idesc_o);
       };
       for (int it = item_lo; it < item_hi && ok; ++it) {
         const WorkItem w = p.items[it];
@@ -208,15 +245,19 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const AttnParams 
           const uint32_t st = (kt + j) % KV_STAGES, ph = ((kt + j) / KV_STAGES) & 1;
           const uint32_t st1 = (kt + j + 1) % KV_STAGES, ph1 = ((kt + j + 1) / KV_STAGES) & 1;
           if (!(ok = mbar_wait(&bar_v_full[st], ph, abortp, p.status, 23))) break;
+          HC_STAMP(kt + j, 2);
           for (int t = 0; t < n_q && ok; ++t) {
             if (!(ok = mbar_wait(&bar_p_full[t], p_cnt[t] & 1, abortp, p.status, 24))) break;
+            HC_STAMP(kt + j, 3 + 3 * t);
             ++p_cnt[t];
             tc_fence_after_sync();
             issue_pv(t, st, j > 0);
             if (j + 1 < nt) {
               if (t == 0 && !(ok = mbar_wait(&bar_k_full[st1], ph1, abortp, p.status, 25))) break;
+              HC_STAMP(kt + j, 4 + 3 * t);
               tc_fence_after_sync();
               issue_qk(t, st1);
+              HC_STAMP(kt + j, 5 + 3 * t);
               mma_commit(&bar_s_full[t]);
               if (t == n_q - 1) mma_commit(&bar_k_free[st1]);
             } else {
@@ -229,9 +270,9 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const AttnParams 
         kt += nt;
       }
     }
-  } else {
+  } else if (warp >= 4) {
     // ------------------------------------------------------------------ softmax + epilogue warpgroups
-    const int t = (warp - 2) >> 2;                  // query tile of this warpgroup
+    const int t = (warp - 4) >> 2;                  // query tile of this warpgroup
     const int r = ((warp & 3) << 5) | lane;         // row inside the tile == TMEM lane
     const uint32_t lane_off = static_cast<uint32_t>((warp & 3) << 5) << 16;
     const uint32_t s_addr = tmem + lane_off + S_COL + t * 128;
@@ -242,6 +283,7 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const AttnParams 
     for (int it = item_lo; it < item_hi && ok; ++it) {
       const WorkItem w = p.items[it];
       if (w.q_count[t] == 0) continue;
+      if (p.trace && t == 0 && r == 0) p.trace[2 * it] = global_timer_ns();
       const bool row_valid = r < w.q_count[t];
       int token = 0;
       if (row_valid) {
@@ -275,33 +317,41 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const AttnParams 
         const int n_valid = min(128, w.seg_len - c * 128);
         const int tok0 = PROXY ? (w.kv_row0 + c * 128) : 0;  // in-frame token of this tile's first key
         if (!(ok = mbar_wait(&bar_s_full[t], s_cnt & 1, abortp, p.status, 31))) break;
+        if (r == 0) HC_STAMP(s_cnt, 9 + 3 * t);
         ++s_cnt;
         tc_fence_after_sync();
-        // pass 1: row maximum of the raw logits
-        float mx = -INFINITY;
-#pragma unroll 1
-        for (int ch = 0; ch < 4; ++ch) {
-          uint32_t v[32];
-          tmem_ld32(s_addr + ch * 32, v);
-          tmem_wait_ld();
-          if (PROXY) {
-            int ky = (tok0 + ch * 32) / p.grid_w, kx = (tok0 + ch * 32) - ky * p.grid_w;
+        // the whole logit row of this thread: 128 fp32 values, loaded with four back-to-back TMEM reads
+        uint32_t sv[128];
 #pragma unroll
-            for (int i = 0; i < 32; ++i) {
-              const bool a = (ch * 32 + i < n_valid) && (abs(ky - qy) <= p.radius) && (abs(kx - qx) <= p.radius);
-              if (a) mx = fmaxf(mx, __uint_as_float(v[i]));
-              if (++kx == p.grid_w) { kx = 0; ++ky; }
-            }
-          } else if (ch * 32 + 32 <= n_valid) {
+        for (int ch = 0; ch < 4; ++ch) tmem_ld32(s_addr + ch * 32, reinterpret_cast<uint32_t(&)[32]>(sv[ch * 32]));
+        tmem_wait_ld();
+        if (r == 0) HC_STAMP(s_cnt - 1, 10 + 3 * t);
+        // keys this row must not see get a logit of -inf: the ragged tail of a segment, and for the
+        // Spatial proxy every key outside the (2r+1)^2 neighbourhood of the query's grid position
+        if (PROXY) {
+          int ky = tok0 / p.grid_w, kx = tok0 - ky * p.grid_w;
 #pragma unroll
-            for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(v[i]));
-          } else {
-#pragma unroll
-            for (int i = 0; i < 32; ++i)
-              if (ch * 32 + i < n_valid) mx = fmaxf(mx, __uint_as_float(v[i]));
+          for (int i = 0; i < 128; ++i) {
+            const bool a = (i < n_valid) && (abs(ky - qy) <= p.radius) && (abs(kx - qx) <= p.radius);
+            if (!a) sv[i] = 0xff800000u;
+            if (++kx == p.grid_w) { kx = 0; ++ky; }
           }
+        } else if (n_valid < 128) {
+#pragma unroll
+          for (int i = 0; i < 128; ++i)
+            if (i >= n_valid) sv[i] = 0xff800000u;
         }
+        float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+        for (int i = 0; i < 128; i += 8) {
+          mx4[0] = max3(mx4[0], __uint_as_float(sv[i]), __uint_as_float(sv[i + 1]));
+          mx4[1] = max3(mx4[1], __uint_as_float(sv[i + 2]), __uint_as_float(sv[i + 3]));
+          mx4[2] = max3(mx4[2], __uint_as_float(sv[i + 4]), __uint_as_float(sv[i + 5]));
+          mx4[3] = max3(mx4[3], __uint_as_float(sv[i + 6]), __uint_as_float(sv[i + 7]));
+        }
+        float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
         mx *= p.scale_log2e;  // scale > 0, so the maximum commutes with it
+        if (r == 0 && t == 0) HC_STAMP(s_cnt - 1, 15);
         // running maximum: move the reference only when some row of the warp outgrew it by 2^8
         const bool grow = mx > m_ref + RESCALE_THRESHOLD || (m_ref == -INFINITY && mx > -INFINITY);
         if (__any_sync(0xffffffffu, grow)) {
@@ -323,44 +373,48 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const AttnParams 
           }
         }
         const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
-        // pass 2: p = 2^(s * c - m), row sum, bf16 pack into the first 64 columns of S_t
-        float tile_sum = 0.f;
-#pragma unroll 1
+        if (r == 0 && t == 0) HC_STAMP(s_cnt - 1, 7);
+        // p = 2^(s * c - m) for two keys per special-function operation, row sum in fp32, bf16 pack into the
+        // first 64 columns of S_t
+        const uint64_t c2 = pack_f32x2(p.scale_log2e, p.scale_log2e), m2 = pack_f32x2(-m_use, -m_use);
+        uint64_t sum2[2] = {0ull, 0ull};
+#pragma unroll
         for (int ch = 0; ch < 4; ++ch) {
-          uint32_t v[32];
-          tmem_ld32(s_addr + ch * 32, v);
-          tmem_wait_ld();
-          float e[32];
-          if (PROXY) {
-            int ky = (tok0 + ch * 32) / p.grid_w, kx = (tok0 + ch * 32) - ky * p.grid_w;
-#pragma unroll
-            for (int i = 0; i < 32; ++i) {
-              const bool a = (ch * 32 + i < n_valid) && (abs(ky - qy) <= p.radius) && (abs(kx - qx) <= p.radius);
-              e[i] = a ? ex2_approx(fmaf(__uint_as_float(v[i]), p.scale_log2e, -m_use)) : 0.f;
-              if (++kx == p.grid_w) { kx = 0; ++ky; }
-            }
-          } else if (ch * 32 + 32 <= n_valid) {
-#pragma unroll
-            for (int i = 0; i < 32; ++i) e[i] = ex2_approx(fmaf(__uint_as_float(v[i]), p.scale_log2e, -m_use));
-          } else {
-#pragma unroll
-            for (int i = 0; i < 32; ++i)
-              e[i] = (ch * 32 + i < n_valid) ? ex2_approx(fmaf(__uint_as_float(v[i]), p.scale_log2e, -m_use)) : 0.f;
-          }
           uint32_t pk[16];
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
-            tile_sum += e[2 * i] + e[2 * i + 1];
-            pk[i] = pack_bf16x2(e[2 * i], e[2 * i + 1]);
+            const uint64_t x2 = fma_f32x2(
+                pack_f32x2(__uint_as_float(sv[ch * 32 + 2 * i]), __uint_as_float(sv[ch * 32 + 2 * i + 1])), c2, m2);
+            float x0, x1, e0, e1;
+            unpack_f32x2(x2, x0, x1);
+#if HC_EXP_MODE == 0
+            e0 = ex2_approx(x0);
+            e1 = ex2_approx(x1);
+            pk[i] = pack_bf16x2(e0, e1);
+#elif HC_EXP_MODE == 1
+            ex2_pair(x0, x1, e0, e1);
+            pk[i] = pack_bf16x2(e0, e1);
+#else
+            pk[i] = (HC_EXP_MODE == 2) ? ex2_pair_bf16_cvt(x0, x1) : ex2_pair_bf16(x0, x1);
+            e0 = __uint_as_float(pk[i] << 16);
+            e1 = __uint_as_float(pk[i] & 0xffff0000u);
+#endif
+            sum2[i & 1] = add_f32x2(sum2[i & 1], pack_f32x2(e0, e1));
           }
           tmem_st16(s_addr + ch * 16, pk);
         }
+        if (r == 0 && t == 0) HC_STAMP(s_cnt - 1, 8);
+        float t0, t1, t2, t3;
+        unpack_f32x2(sum2[0], t0, t1);
+        unpack_f32x2(sum2[1], t2, t3);
+        const float tile_sum = (t0 + t1) + (t2 + t3);
         l_sum += tile_sum;
         if (PROXY && seg >= p.mid_seg_lo && seg < p.mid_seg_hi && !(seg >= p.last_seg_lo && seg < p.last_seg_hi))
           l_mid += tile_sum;
         tmem_wait_st();
         tc_fence_before_sync();
         mbar_arrive(&bar_p_full[t]);
+        if (r == 0) HC_STAMP(s_cnt - 1, 11 + 3 * t);
       }
       if (!ok) break;
       // ---- epilogue
@@ -409,6 +463,7 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const AttnParams 
           if (PROXY) p.f32_lse[(w.out_slot + 1) * lh + idx] = (l_mid > 0.f) ? m_ref * ln2 + __logf(l_mid) : -INFINITY;
         }
       }
+      if (p.trace && t == 0 && r == 0) p.trace[2 * it + 1] = global_timer_ns();
     }
   }
   // ------------------------------------------------------------------ teardown
@@ -421,45 +476,48 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const AttnParams 
 }
 
 // Merges the partial results of query tiles whose key range was cut into several work items:
-// out = sum_i 2^(m_i - m) O_i / sum_i 2^(m_i - m) l_i.  One thread per (row, 8 output columns).
+// out = sum_i 2^(m_i - m) O_i / sum_i 2^(m_i - m) l_i.  One thread per (row, 8 output columns),
+// COMBINE_ROWS rows per block.
 struct CombineEntry {
   int32_t head, cell, q_start, q_count;  // one 128-row query tile
   int32_t first_slot, n_parts, sub;      // partial slots first_slot .. +n_parts-1, rows sub*128 .. of each slot
   int32_t pad;
 };
 
+constexpr int COMBINE_ROWS = 16;  // query rows per block of combine_kernel
+
 template <int D>
-__global__ void combine_kernel(const CombineEntry* entries, const CellGeom* cells, const float* part_o,
-                               const float2* part_ml, __nv_bfloat16* out, int n_heads, int tokens_per_frame,
-                               int grid_w) {
-  const CombineEntry e = entries[blockIdx.x];
+__global__ void __launch_bounds__(COMBINE_ROWS * (D / 8))
+combine_kernel(const CombineEntry* entries, const CellGeom* cells, const float* part_o, const float2* part_ml,
+               __nv_bfloat16* out, int n_heads, int tokens_per_frame, int grid_w) {
   constexpr int CHUNKS = D / 8;
-  for (int idx = threadIdx.x; idx < e.q_count * CHUNKS; idx += blockDim.x) {
-    const int r = idx / CHUNKS, c = idx - r * CHUNKS;
-    float m = -INFINITY;
-    for (int i = 0; i < e.n_parts; ++i)
-      m = fmaxf(m, part_ml[static_cast<size_t>(e.first_slot + i) * 256 + e.sub * 128 + r].x);
-    float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0}, l = 0.f;
-    for (int i = 0; i < e.n_parts; ++i) {
-      const size_t row = static_cast<size_t>(e.first_slot + i) * 256 + e.sub * 128 + r;
-      const float2 ml = part_ml[row];
-      const float wgt = (ml.x == -INFINITY) ? 0.f : ex2_approx(ml.x - m);
-      l += wgt * ml.y;
-      const float4* src = reinterpret_cast<const float4*>(part_o + row * D + c * 8);
-      const float4 a = src[0], b = src[1];
-      acc[0] += wgt * a.x; acc[1] += wgt * a.y; acc[2] += wgt * a.z; acc[3] += wgt * a.w;
-      acc[4] += wgt * b.x; acc[5] += wgt * b.y; acc[6] += wgt * b.z; acc[7] += wgt * b.w;
-    }
-    const float inv = l > 0.f ? 1.f / l : 0.f;
-    int token = e.q_start + r;
-    if (e.cell >= 0) token = cell_query_token(cells[e.cell], token, tokens_per_frame, grid_w);
-    uint4 o4;
-    o4.x = pack_bf16x2(acc[0] * inv, acc[1] * inv);
-    o4.y = pack_bf16x2(acc[2] * inv, acc[3] * inv);
-    o4.z = pack_bf16x2(acc[4] * inv, acc[5] * inv);
-    o4.w = pack_bf16x2(acc[6] * inv, acc[7] * inv);
-    *reinterpret_cast<uint4*>(out + (static_cast<size_t>(token) * n_heads + e.head) * D + c * 8) = o4;
+  const CombineEntry e = entries[blockIdx.x / (128 / COMBINE_ROWS)];
+  const int r = (blockIdx.x % (128 / COMBINE_ROWS)) * COMBINE_ROWS + threadIdx.x / CHUNKS;
+  const int c = threadIdx.x % CHUNKS;
+  if (r >= e.q_count) return;
+  float m = -INFINITY;
+  for (int i = 0; i < e.n_parts; ++i)
+    m = fmaxf(m, part_ml[static_cast<size_t>(e.first_slot + i) * 256 + e.sub * 128 + r].x);
+  float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0}, l = 0.f;
+  for (int i = 0; i < e.n_parts; ++i) {
+    const size_t row = static_cast<size_t>(e.first_slot + i) * 256 + e.sub * 128 + r;
+    const float2 ml = part_ml[row];
+    const float wgt = (ml.x == -INFINITY) ? 0.f : ex2_approx(ml.x - m);
+    l += wgt * ml.y;
+    const float4* src = reinterpret_cast<const float4*>(part_o + row * D + c * 8);
+    const float4 a = src[0], b = src[1];
+    acc[0] += wgt * a.x; acc[1] += wgt * a.y; acc[2] += wgt * a.z; acc[3] += wgt * a.w;
+    acc[4] += wgt * b.x; acc[5] += wgt * b.y; acc[6] += wgt * b.z; acc[7] += wgt * b.w;
   }
+  const float inv = l > 0.f ? 1.f / l : 0.f;
+  int token = e.q_start + r;
+  if (e.cell >= 0) token = cell_query_token(cells[e.cell], token, tokens_per_frame, grid_w);
+  uint4 o4;
+  o4.x = pack_bf16x2(acc[0] * inv, acc[1] * inv);
+  o4.y = pack_bf16x2(acc[2] * inv, acc[3] * inv);
+  o4.z = pack_bf16x2(acc[4] * inv, acc[5] * inv);
+  o4.w = pack_bf16x2(acc[6] * inv, acc[7] * inv);
+  *reinterpret_cast<uint4*>(out + (static_cast<size_t>(token) * n_heads + e.head) * D + c * 8) = o4;
 }
 
 }  // namespace hc

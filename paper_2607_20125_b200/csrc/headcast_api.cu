@@ -7,6 +7,7 @@
 #include <cmath>
 #include <cstdarg>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <queue>
 #include <string>
@@ -93,6 +94,13 @@ struct headcast_ctx {
 
   int n_sm = 148;
   int64_t launches = 0;
+  bool tracing = false;  // record per-item start/end times in the attention kernel
+  DevBuf<unsigned long long> trace_dev;
+  std::vector<WorkItem> trace_items;
+  std::vector<int32_t> trace_cta_first;
+  bool timing = false;  // record events around the attention kernel of each call
+  cudaEvent_t ev_a = nullptr, ev_b = nullptr;
+  bool ev_valid = false;
   std::string err;
 };
 
@@ -206,67 +214,100 @@ WorkItem range_item(int head, int map, int x0, long long row0, int n_keys) {
   return w;
 }
 
-constexpr double ITEM_OVERHEAD = 3.0;  // tile-times charged per item for the query load, pipeline fill and epilogue
+constexpr double ITEM_OVERHEAD = 4.0;  // tile-times charged per item for the query load, pipeline fill and epilogue
+constexpr int MIN_PART_TILES = 4;      // never cut a key range into pieces shorter than this
 
 double item_cost(const WorkItem& w) {
   const int n_q = w.q_count[1] > 0 ? 2 : 1;
   return static_cast<double>(n_q) * (w.tile_end - w.tile_begin) + ITEM_OVERHEAD;
 }
 
-// Cuts long items along the key range (partials merged by combine_kernel), then assigns items to CTAs
-// longest-first onto the least loaded CTA.
+// Assigns work to the persistent CTAs (one per SM).
+//  - allow_split: the items, longest first, are laid end to end and the line is cut into one equal share per
+//    CTA; an item that straddles a cut is divided along its key range, its pieces write unnormalised partial
+//    results and combine_kernel merges them.  Every CTA then carries the same number of tile-times.
+//  - otherwise (outputs that cannot be merged afterwards): whole items, longest first, onto the least loaded CTA.
 void finalize_schedule(headcast_ctx* c, Schedule& s, std::vector<Proto>& protos, bool allow_split) {
   s.items.clear();
   s.combine.clear();
   s.n_slots = 0;
-  double total = 0.0;
-  for (const Proto& p : protos) total += item_cost(p.w);
-  const double max_cost = std::max(48.0, total / c->n_sm / 2.5);
-  std::vector<WorkItem> all;
-  for (const Proto& p : protos) {
-    const int n_q = p.w.q_count[1] > 0 ? 2 : 1;
-    int parts = 1;
-    if (allow_split) parts = std::max(1, static_cast<int>(std::ceil(item_cost(p.w) / max_cost)));
-    parts = std::min(parts, p.n_tiles);
-    if (parts == 1) {
-      all.push_back(p.w);
-      continue;
-    }
-    const int per = (p.n_tiles + parts - 1) / parts;
-    const int first_slot = s.n_slots;
-    int made = 0;
-    for (int b = 0; b < p.n_tiles; b += per, ++made) {
-      WorkItem w = p.w;
-      w.tile_begin = b;
-      w.tile_end = std::min(p.n_tiles, b + per);
-      w.out_mode = OUT_PARTIAL;
-      w.out_slot = s.n_slots++;
-      all.push_back(w);
-    }
-    for (int t = 0; t < n_q; ++t) {
-      CombineEntry e;
-      e.head = p.w.head;
-      e.cell = p.w.cell;
-      e.q_start = p.w.q_start[t];
-      e.q_count = p.w.q_count[t];
-      e.first_slot = first_slot;
-      e.n_parts = made;
-      e.sub = t;
-      e.pad = 0;
-      s.combine.push_back(e);
-    }
-  }
-  std::stable_sort(all.begin(), all.end(), [](const WorkItem& a, const WorkItem& b) { return item_cost(a) > item_cost(b); });
   const int n_cta = c->n_sm;
   std::vector<std::vector<WorkItem>> bins(n_cta);
-  typedef std::pair<double, int> Load;
-  std::priority_queue<Load, std::vector<Load>, std::greater<Load>> pq;
-  for (int b = 0; b < n_cta; ++b) pq.push(Load(0.0, b));
-  for (const WorkItem& w : all) {
-    Load l = pq.top();
-    pq.pop();
-    bins[l.second].push_back(w);
-    pq.push(Load(l.first + item_cost(w), l.second));
+  std::stable_sort(protos.begin(), protos.end(),
+                   [](const Proto& a, const Proto& b) { return item_cost(a.w) > item_cost(b.w); });
+  if (allow_split) {
+    double total = 0.0;
+    for (const Proto& p : protos) total += item_cost(p.w);
+    const double slack = 0.02 * total / n_cta;
+    int cta = 0;
+    double unassigned = total;  // tile-times not yet placed; the share of each further CTA is re-derived from it
+    double room = total / n_cta;
+    auto next_cta = [&]() {
+      if (cta + 1 < n_cta) {
+        ++cta;
+        room = unassigned / (n_cta - cta);
+      } else {
+        room = 1e30;
+      }
+    };
+    for (const Proto& p : protos) {
+      const int n_q = p.w.q_count[1] > 0 ? 2 : 1;
+      std::vector<std::pair<int, WorkItem>> parts;  // (cta, piece)
+      int begin = 0;
+      while (begin < p.n_tiles) {
+        const int left = p.n_tiles - begin;
+        const double need = static_cast<double>(n_q) * left + ITEM_OVERHEAD;
+        int take = left;
+        if (need > room + slack) {
+          const int can = static_cast<int>(std::floor((room - ITEM_OVERHEAD) / n_q));
+          if (can < MIN_PART_TILES) {
+            next_cta();
+            continue;
+          }
+          if (left - can >= MIN_PART_TILES) take = can;
+        }
+        WorkItem w = p.w;
+        w.tile_begin = begin;
+        w.tile_end = begin + take;
+        parts.push_back(std::make_pair(cta, w));
+        room -= static_cast<double>(n_q) * take + ITEM_OVERHEAD;
+        unassigned -= static_cast<double>(n_q) * take + (begin == 0 ? ITEM_OVERHEAD : 0.0);
+        begin += take;
+        if (room < ITEM_OVERHEAD + MIN_PART_TILES) next_cta();
+      }
+      if (parts.size() == 1) {
+        bins[parts[0].first].push_back(parts[0].second);
+        continue;
+      }
+      const int first_slot = s.n_slots;
+      for (auto& pr : parts) {
+        pr.second.out_mode = OUT_PARTIAL;
+        pr.second.out_slot = s.n_slots++;
+        bins[pr.first].push_back(pr.second);
+      }
+      for (int t = 0; t < n_q; ++t) {
+        CombineEntry e;
+        e.head = p.w.head;
+        e.cell = p.w.cell;
+        e.q_start = p.w.q_start[t];
+        e.q_count = p.w.q_count[t];
+        e.first_slot = first_slot;
+        e.n_parts = static_cast<int32_t>(parts.size());
+        e.sub = t;
+        e.pad = 0;
+        s.combine.push_back(e);
+      }
+    }
+  } else {
+    typedef std::pair<double, int> Load;
+    std::priority_queue<Load, std::vector<Load>, std::greater<Load>> pq;
+    for (int b = 0; b < n_cta; ++b) pq.push(Load(0.0, b));
+    for (const Proto& p : protos) {
+      Load l = pq.top();
+      pq.pop();
+      bins[l.second].push_back(p.w);
+      pq.push(Load(l.first + item_cost(p.w), l.second));
+    }
   }
   s.cta_first.assign(n_cta + 1, 0);
   for (int b = 0; b < n_cta; ++b) {
@@ -353,8 +394,13 @@ int launch_attn_t(headcast_ctx* c, const AttnParams& p, cudaStream_t st) {
                                     AttnSmem<D>::DYN_BYTES));
     configured = true;
   }
+  if (c->timing) HC_CUDA(c, cudaEventRecord(c->ev_a, st));
   attn_kernel<D, PROXY><<<c->n_sm, ATTN_THREADS, AttnSmem<D>::DYN_BYTES, st>>>(p);
   HC_CUDA(c, cudaGetLastError());
+  if (c->timing) {
+    HC_CUDA(c, cudaEventRecord(c->ev_b, st));
+    c->ev_valid = true;
+  }
   ++c->launches;
   return HC_OK;
 }
@@ -381,6 +427,15 @@ int run_schedule(headcast_ctx* c, Schedule& s, const void* q, void* out, bool pr
   p.block_tokens = c->L;
   p.scale_log2e = c->scale * 1.4426950408889634f;
   p.status = c->status_dev;
+  p.trace = nullptr;
+  if (c->tracing) {
+    HC_CUDA(c, c->trace_dev.reserve(2 * s.items.size() + 16 * 64));
+    HC_CUDA(c, cudaMemsetAsync(c->trace_dev.ptr, 0, (2 * s.items.size() + 16 * 64) * sizeof(unsigned long long), st));
+    p.trace = c->trace_dev.ptr;
+    p.trace_base = static_cast<int32_t>(2 * s.items.size());
+    c->trace_items = s.items;
+    c->trace_cta_first = s.cta_first;
+  }
   p.radius = c->cfg.proxy_radius;
   if (proxy) {
     const int newest = c->slots.back();
@@ -395,12 +450,13 @@ int run_schedule(headcast_ctx* c, Schedule& s, const void* q, void* out, bool pr
     rc = proxy ? launch_attn_t<64, true>(c, p, st) : launch_attn_t<64, false>(c, p, st);
   if (rc != HC_OK) return rc;
   if (!s.combine.empty()) {
+    const unsigned blocks = static_cast<unsigned>(s.combine.size()) * (128 / COMBINE_ROWS);
     if (c->D == 128)
-      combine_kernel<128><<<static_cast<unsigned>(s.combine.size()), 256, 0, st>>>(
-          s.combine_dev.ptr, c->cells_dev, c->part_o.ptr, c->part_ml.ptr, p.out, c->H, c->T_f, c->G_w);
+      combine_kernel<128><<<blocks, COMBINE_ROWS * 16, 0, st>>>(s.combine_dev.ptr, c->cells_dev, c->part_o.ptr,
+                                                                c->part_ml.ptr, p.out, c->H, c->T_f, c->G_w);
     else
-      combine_kernel<64><<<static_cast<unsigned>(s.combine.size()), 256, 0, st>>>(
-          s.combine_dev.ptr, c->cells_dev, c->part_o.ptr, c->part_ml.ptr, p.out, c->H, c->T_f, c->G_w);
+      combine_kernel<64><<<blocks, COMBINE_ROWS * 8, 0, st>>>(s.combine_dev.ptr, c->cells_dev, c->part_o.ptr,
+                                                              c->part_ml.ptr, p.out, c->H, c->T_f, c->G_w);
     HC_CUDA(c, cudaGetLastError());
     ++c->launches;
   }
@@ -547,6 +603,9 @@ int headcast_create(const headcast_config* cfg, headcast_ctx** out) {
     return HC_ERR_UNSUPPORTED;
   }
   c->n_sm = prop.multiProcessorCount;
+#ifdef HC_TIMELINE
+  if (const char* e = getenv("HEADCAST_NUM_CTAS")) c->n_sm = std::max(1, atoi(e));
+#endif
   const size_t mono_bytes = cache_elems(c, c->H) * sizeof(__nv_bfloat16);
   cudaError_t e = cudaSuccess;
   auto step = [&](cudaError_t r) { if (e == cudaSuccess) e = r; };
@@ -584,12 +643,15 @@ int headcast_destroy(headcast_ctx* c) {
                   c->sp_base, c->sp_nc, c->cells_dev, c->maps_dev, c->status_dev};
   for (void* p : ptrs)
     if (p) cudaFree(p);
+  if (c->ev_a) cudaEventDestroy(c->ev_a);
+  if (c->ev_b) cudaEventDestroy(c->ev_b);
   c->sched_dense.release();
   c->sched_hc.release();
   c->sched_cls.release();
   c->sched_proxy.release();
   c->part_o.release();
   c->part_ml.release();
+  c->trace_dev.release();
   c->cls_o.release();
   c->cls_lse.release();
   c->cls_tok.release();
@@ -881,6 +943,66 @@ double headcast_attend_flops(const headcast_ctx* c, int32_t dense) {
   }
   return f;
 }
+
+int headcast_set_kernel_timing(headcast_ctx* c, int32_t enable) {
+  if (!c) return HC_ERR_INVALID_ARG;
+  if (enable && !c->ev_a) {
+    HC_CUDA(c, cudaEventCreate(&c->ev_a));
+    HC_CUDA(c, cudaEventCreate(&c->ev_b));
+  }
+  c->timing = enable != 0;
+  c->ev_valid = false;
+  return HC_OK;
+}
+
+int headcast_last_attention_kernel_ms(headcast_ctx* c, float* ms_host) {
+  if (!c || !ms_host) return HC_ERR_INVALID_ARG;
+  if (!c->ev_valid) return fail(c, HC_ERR_STATE, "no attention kernel was timed yet");
+  HC_CUDA(c, cudaEventSynchronize(c->ev_b));
+  HC_CUDA(c, cudaEventElapsedTime(ms_host, c->ev_a, c->ev_b));
+  return HC_OK;
+}
+
+int headcast_set_tracing(headcast_ctx* c, int32_t enable) {
+  if (!c) return HC_ERR_INVALID_ARG;
+  c->tracing = enable != 0;
+  return HC_OK;
+}
+
+int headcast_read_trace(headcast_ctx* c, int64_t* rows_host, int32_t capacity, int32_t* n_items_host) {
+  if (!c || !n_items_host) return HC_ERR_INVALID_ARG;
+  const int n = static_cast<int>(c->trace_items.size());
+  *n_items_host = n;
+  if (!rows_host || n == 0) return HC_OK;
+  HC_CUDA(c, cudaDeviceSynchronize());
+  std::vector<unsigned long long> t(2 * static_cast<size_t>(n));
+  HC_CUDA(c, cudaMemcpy(t.data(), c->trace_dev.ptr, t.size() * sizeof(unsigned long long), cudaMemcpyDeviceToHost));
+  int cta = 0;
+  for (int i = 0; i < n && i < capacity; ++i) {
+    while (cta + 1 < static_cast<int>(c->trace_cta_first.size()) && c->trace_cta_first[cta + 1] <= i) ++cta;
+    const WorkItem& w = c->trace_items[i];
+    int64_t* r = rows_host + 8 * static_cast<size_t>(i);
+    r[0] = cta;
+    r[1] = w.head;
+    r[2] = w.cell;
+    r[3] = w.q_count[0] + w.q_count[1];
+    r[4] = w.tile_end - w.tile_begin;
+    r[5] = w.out_mode;
+    r[6] = static_cast<int64_t>(t[2 * i]);
+    r[7] = static_cast<int64_t>(t[2 * i + 1]);
+  }
+  return HC_OK;
+}
+
+#ifdef HC_TIMELINE
+int headcast_read_timeline(headcast_ctx* c, int64_t* out_host /* [64][16] */) {
+  if (!c || !out_host || c->trace_items.empty()) return HC_ERR_INVALID_ARG;
+  HC_CUDA(c, cudaDeviceSynchronize());
+  HC_CUDA(c, cudaMemcpy(out_host, c->trace_dev.ptr + 2 * c->trace_items.size(), 16 * 64 * sizeof(int64_t),
+                        cudaMemcpyDeviceToHost));
+  return HC_OK;
+}
+#endif
 
 int headcast_check(headcast_ctx* c, void* stream) {
   if (!c) return HC_ERR_INVALID_ARG;
