@@ -130,7 +130,8 @@ def _oracle_state(w):
             cache.append(*synth.make_kv(w, b))
         cache.split(w.labels)
         q = synth.make_q(w, w.n_blocks - 1, 0)
-        rows = synth.sample_rows(w, n_random=64)
+        rows = synth.sample_rows(w, n_random=4096)
+        rows = rows[np.random.default_rng(0).permutation(rows.size)]
         t0 = time.perf_counter()
         orc.attend(q, cache, geom, rows=rows[:32])
         per_row = (time.perf_counter() - t0) / 32

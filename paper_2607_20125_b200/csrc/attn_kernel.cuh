@@ -7,8 +7,8 @@
 //     product straight from tensor memory);
 //   - K/V tiles (128 keys) arrive through TMA into a 2-stage shared-memory ring (128-byte swizzle);
 //   - two softmax warpgroups, one per query tile, own one query row per thread (online softmax in the
-//     exp2 domain, two exponentials per special-function operation through packed fp16, rescaling of O
-//     only when the running maximum grew by more than 2^8);
+//     exp2 domain, a quarter of the exponentials evaluated as a cubic on the FMA pipe to relieve the
+//     special-function unit, rescaling of O only when the running maximum grew by more than 2^8);
 //   - warp 0 is the TMA producer, warp 1 issues every MMA.
 // Which keys a query tile sees is entirely a property of the work item: a row range of one of the
 // cache buffers (whole window, one block, one Spatial cell) or, for the classification's Spatial
@@ -20,17 +20,6 @@
 #include "tc05.cuh"
 
 namespace hc {
-
-// Development aid (compile with -DHC_TIMELINE): CTA 0 stamps the global timer at the hand-over points of
-// its first key tiles into AttnParams::trace (which must then hold 16 * 64 values beyond the per-item area).
-#ifdef HC_TIMELINE
-#define HC_STAMP(iter, slot)                                                                     \
-  do {                                                                                           \
-    if (p.trace && blockIdx.x == 0 && (iter) < 64) p.trace[p.trace_base + (iter) * 16 + (slot)] = global_timer_ns(); \
-  } while (0)
-#else
-#define HC_STAMP(iter, slot) do { } while (0)
-#endif
 
 struct CellGeom {
   int32_t y0, x0, ch, cw;  // top-left grid position and extent of a deployed Spatial cell
@@ -69,7 +58,6 @@ struct AttnParams {
   int32_t n_heads, tokens_per_frame, grid_w, block_tokens;
   float scale_log2e;       // softmax scale * log2(e)
   int32_t* status;
-  int32_t trace_base;
   unsigned long long* trace;  // optional [2 * n_items]: globaltimer (ns) when query tile 0's warpgroup starts / ends an item
   // Spatial proxy only
   int32_t radius;
@@ -78,9 +66,6 @@ struct AttnParams {
 
 constexpr int ATTN_THREADS = 384;  // warp 0: TMA, warp 1: MMA, warps 2-3 idle, warps 4-7 / 8-11: softmax for query tile 0 / 1
 constexpr int KV_STAGES = 2;
-#ifndef HC_EXP_MODE
-#define HC_EXP_MODE 1
-#endif
 #ifndef HC_RESCALE_THRESHOLD
 #define HC_RESCALE_THRESHOLD 8.0f
 #endif
@@ -110,8 +95,7 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const AttnParams 
   using SM = AttnSmem<D>;
   constexpr int NB = D / 64;          // 64-column blocks per tile
   constexpr int QK_STEPS = D / 16;    // k-steps of S = Q K^T
-  constexpr int PV_STEPS = 128 / 16;  // k-steps of O += P V
-  constexpr uint32_t TMEM_COLS = 512;
+    constexpr uint32_t TMEM_COLS = 512;
   constexpr uint32_t S_COL = 0, O_COL = 256;  // S_t at t*128, O_t at 256 + t*128; P_t overlays S_t
 
   extern __shared__ uint8_t smem_raw[];
@@ -164,13 +148,11 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const AttnParams 
           const int row = w.kv_row0 + seg * w.seg_stride + c * 128;
           const uint32_t st = kt % KV_STAGES, ph = (kt / KV_STAGES) & 1;
           if (!(ok = mbar_wait(&bar_k_free[st], ph ^ 1, abortp, p.status, 11))) break;
-          HC_STAMP(kt, 0);
           mbar_arrive_expect_tx(&bar_k_full[st], SM::TILE_BYTES);
           for (int b = 0; b < NB; ++b)
             tma_load_2d(smem + SM::K_OFF + st * SM::TILE_BYTES + b * SM::BLOCK_BYTES, kmap, w.kv_x0 + 64 * b, row,
                         &bar_k_full[st]);
           if (!(ok = mbar_wait(&bar_v_free[st], ph ^ 1, abortp, p.status, 12))) break;
-          HC_STAMP(kt, 1);
           mbar_arrive_expect_tx(&bar_v_full[st], SM::TILE_BYTES);
           for (int b = 0; b < NB; ++b)
             tma_load_2d(smem + SM::V_OFF + st * SM::TILE_BYTES + b * SM::BLOCK_BYTES, vmap, w.kv_x0 + 64 * b, row,
@@ -196,33 +178,15 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const AttnParams 
                      v_addr = smem_u32(smem + SM::V_OFF);
       uint32_t kt = 0, q_cnt[2] = {0, 0}, p_cnt[2] = {0, 0};
       bool ok = true;
-      // descriptors: the high halves are constant, the low halves are (address >> 4) plus a per-k-step constant
-      const uint32_t kmajor_hi = static_cast<uint32_t>(smem_desc_sw128(0, 16, 1024) >> 32);
-      const uint32_t kmajor_lo = static_cast<uint32_t>(smem_desc_sw128(0, 16, 1024));
-      const uint32_t v_hi = static_cast<uint32_t>(smem_desc_sw128(0, SM::BLOCK_BYTES, 1024) >> 32);
-      const uint32_t v_lo = static_cast<uint32_t>(smem_desc_sw128(0, SM::BLOCK_BYTES, 1024));
+      const uint64_t q_desc = smem_desc_sw128(q_addr, 16, 1024), k_desc = smem_desc_sw128(k_addr, 16, 1024);
+      const uint64_t v_desc = smem_desc_sw128(v_addr, SM::BLOCK_BYTES, 1024);
       auto issue_qk = [&](int t, uint32_t st) {
-        const uint32_t a0 = kmajor_lo + ((q_addr + t * SM::TILE_BYTES) >> 4);
-        const uint32_t b0 = kmajor_lo + ((k_addr + st * SM::TILE_BYTES) >> 4);
-        const uint32_t d = tmem + S_COL + t * 128;
-#pragma unroll
-        for (int kk = 0; kk < QK_STEPS; ++kk) {
-          const uint32_t off = ((kk / 4) * SM::BLOCK_BYTES + (kk % 4) * 32) >> 4;
-          if (kk == 0)
-            mma_ss_lohi<false>(d, a0 + off, kmajor_hi, b0 + off, kmajor_hi, idesc_s);
-          else
-            mma_ss_lohi<true>(d, a0 + off, kmajor_hi, b0 + off, kmajor_hi, idesc_s);
-        }
+        mma_block_ss<QK_STEPS>(tmem + S_COL + t * 128, q_desc + ((t * SM::TILE_BYTES) >> 4),
+                               k_desc + ((st * SM::TILE_BYTES) >> 4), idesc_s, SM::BLOCK_BYTES >> 4, SM::BLOCK_BYTES >> 4);
       };
       auto issue_pv = [&](int t, uint32_t st, bool accumulate) {
-        const uint32_t b0 = v_lo + ((v_addr + st * SM::TILE_BYTES) >> 4);
-        const uint32_t d = tmem + O_COL + t * 128, a = tmem + S_COL + t * 128;
-        if (accumulate)
-          mma_ts_lohi<true>(d, a, b0, v_hi, idesc_o);
-        else
-          mma_ts_lohi<false>(d, a, b0, v_hi, idesc_o);
-#pragma unroll
-        for (int kk = 1; kk < PV_STEPS; ++kk) mma_ts_lohi<true>(d, a + kk * 8, b0 + ((kk * 2048) >> 4), v_hi, idesc_o);
+        mma_block_ts8(tmem + O_COL + t * 128, tmem + S_COL + t * 128, v_desc + ((st * SM::TILE_BYTES) >> 4), idesc_o,
+                      accumulate ? 1u : 0u);
       };
       for (int it = item_lo; it < item_hi && ok; ++it) {
         const WorkItem w = p.items[it];
@@ -245,19 +209,15 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const AttnParams 
           const uint32_t st = (kt + j) % KV_STAGES, ph = ((kt + j) / KV_STAGES) & 1;
           const uint32_t st1 = (kt + j + 1) % KV_STAGES, ph1 = ((kt + j + 1) / KV_STAGES) & 1;
           if (!(ok = mbar_wait(&bar_v_full[st], ph, abortp, p.status, 23))) break;
-          HC_STAMP(kt + j, 2);
           for (int t = 0; t < n_q && ok; ++t) {
             if (!(ok = mbar_wait(&bar_p_full[t], p_cnt[t] & 1, abortp, p.status, 24))) break;
-            HC_STAMP(kt + j, 3 + 3 * t);
             ++p_cnt[t];
             tc_fence_after_sync();
             issue_pv(t, st, j > 0);
             if (j + 1 < nt) {
               if (t == 0 && !(ok = mbar_wait(&bar_k_full[st1], ph1, abortp, p.status, 25))) break;
-              HC_STAMP(kt + j, 4 + 3 * t);
               tc_fence_after_sync();
               issue_qk(t, st1);
-              HC_STAMP(kt + j, 5 + 3 * t);
               mma_commit(&bar_s_full[t]);
               if (t == n_q - 1) mma_commit(&bar_k_free[st1]);
             } else {
@@ -317,7 +277,6 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const AttnParams 
         const int n_valid = min(128, w.seg_len - c * 128);
         const int tok0 = PROXY ? (w.kv_row0 + c * 128) : 0;  // in-frame token of this tile's first key
         if (!(ok = mbar_wait(&bar_s_full[t], s_cnt & 1, abortp, p.status, 31))) break;
-        if (r == 0) HC_STAMP(s_cnt, 9 + 3 * t);
         ++s_cnt;
         tc_fence_after_sync();
         // the whole logit row of this thread: 128 fp32 values, loaded with four back-to-back TMEM reads
@@ -325,7 +284,6 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const AttnParams 
 #pragma unroll
         for (int ch = 0; ch < 4; ++ch) tmem_ld32(s_addr + ch * 32, reinterpret_cast<uint32_t(&)[32]>(sv[ch * 32]));
         tmem_wait_ld();
-        if (r == 0) HC_STAMP(s_cnt - 1, 10 + 3 * t);
         // keys this row must not see get a logit of -inf: the ragged tail of a segment, and for the
         // Spatial proxy every key outside the (2r+1)^2 neighbourhood of the query's grid position
         if (PROXY) {
@@ -351,7 +309,6 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const AttnParams 
         }
         float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
         mx *= p.scale_log2e;  // scale > 0, so the maximum commutes with it
-        if (r == 0 && t == 0) HC_STAMP(s_cnt - 1, 15);
         // running maximum: move the reference only when some row of the warp outgrew it by 2^8
         const bool grow = mx > m_ref + RESCALE_THRESHOLD || (m_ref == -INFINITY && mx > -INFINITY);
         if (__any_sync(0xffffffffu, grow)) {
@@ -373,7 +330,6 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const AttnParams 
           }
         }
         const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
-        if (r == 0 && t == 0) HC_STAMP(s_cnt - 1, 7);
         // p = 2^(s * c - m) for two keys per special-function operation, row sum in fp32, bf16 pack into the
         // first 64 columns of S_t
         const uint64_t c2 = pack_f32x2(p.scale_log2e, p.scale_log2e), m2 = pack_f32x2(-m_use, -m_use);
@@ -387,23 +343,19 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const AttnParams 
                 pack_f32x2(__uint_as_float(sv[ch * 32 + 2 * i]), __uint_as_float(sv[ch * 32 + 2 * i + 1])), c2, m2);
             float x0, x1, e0, e1;
             unpack_f32x2(x2, x0, x1);
-#if HC_EXP_MODE == 0
-            e0 = ex2_approx(x0);
-            e1 = ex2_approx(x1);
+            if ((i & 3) == 3) {
+              // every fourth pair takes the polynomial route on the FMA pipe: the special-function unit alone
+              // cannot produce 128 x 128 exponentials in the time the tensor pipe needs for the tile
+              ex2_poly_pair(pack_f32x2(fmaxf(x0, -126.f), fmaxf(x1, -126.f)), e0, e1);
+            } else {
+              e0 = ex2_approx(x0);
+              e1 = ex2_approx(x1);
+            }
             pk[i] = pack_bf16x2(e0, e1);
-#elif HC_EXP_MODE == 1
-            ex2_pair(x0, x1, e0, e1);
-            pk[i] = pack_bf16x2(e0, e1);
-#else
-            pk[i] = (HC_EXP_MODE == 2) ? ex2_pair_bf16_cvt(x0, x1) : ex2_pair_bf16(x0, x1);
-            e0 = __uint_as_float(pk[i] << 16);
-            e1 = __uint_as_float(pk[i] & 0xffff0000u);
-#endif
             sum2[i & 1] = add_f32x2(sum2[i & 1], pack_f32x2(e0, e1));
           }
           tmem_st16(s_addr + ch * 16, pk);
         }
-        if (r == 0 && t == 0) HC_STAMP(s_cnt - 1, 8);
         float t0, t1, t2, t3;
         unpack_f32x2(sum2[0], t0, t1);
         unpack_f32x2(sum2[1], t2, t3);
@@ -414,7 +366,6 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const AttnParams 
         tmem_wait_st();
         tc_fence_before_sync();
         mbar_arrive(&bar_p_full[t]);
-        if (r == 0) HC_STAMP(s_cnt - 1, 11 + 3 * t);
       }
       if (!ok) break;
       // ---- epilogue

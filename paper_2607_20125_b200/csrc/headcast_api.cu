@@ -214,12 +214,19 @@ WorkItem range_item(int head, int map, int x0, long long row0, int n_keys) {
   return w;
 }
 
-constexpr double ITEM_OVERHEAD = 4.0;  // tile-times charged per item for the query load, pipeline fill and epilogue
-constexpr int MIN_PART_TILES = 4;      // never cut a key range into pieces shorter than this
+// Cost model of the scheduler, in units of the time one key tile takes with both query tiles in flight
+// (fitted to per-item timings from headcast_read_trace on B200): a lone query tile still needs 0.8 of that
+// because the chain S -> softmax -> P -> next S is latency bound; every item pays for its query load, pipeline
+// fill and epilogue; a partial result costs an extra round trip through global memory.
+constexpr double TILE_COST_PAIR = 1.0, TILE_COST_SINGLE = 0.8;
+constexpr double ITEM_OVERHEAD = 3.5;
+constexpr double PARTIAL_EXTRA = 1.0;
+constexpr int MIN_PART_TILES = 4;  // never cut a key range into pieces shorter than this
+
+double tile_cost(const WorkItem& w) { return w.q_count[1] > 0 ? TILE_COST_PAIR : TILE_COST_SINGLE; }
 
 double item_cost(const WorkItem& w) {
-  const int n_q = w.q_count[1] > 0 ? 2 : 1;
-  return static_cast<double>(n_q) * (w.tile_end - w.tile_begin) + ITEM_OVERHEAD;
+  return tile_cost(w) * (w.tile_end - w.tile_begin) + ITEM_OVERHEAD + (w.out_mode == OUT_PARTIAL ? PARTIAL_EXTRA : 0.0);
 }
 
 // Assigns work to the persistent CTAs (one per SM).
@@ -252,14 +259,15 @@ void finalize_schedule(headcast_ctx* c, Schedule& s, std::vector<Proto>& protos,
     };
     for (const Proto& p : protos) {
       const int n_q = p.w.q_count[1] > 0 ? 2 : 1;
+      const double per_tile = tile_cost(p.w);
       std::vector<std::pair<int, WorkItem>> parts;  // (cta, piece)
       int begin = 0;
       while (begin < p.n_tiles) {
         const int left = p.n_tiles - begin;
-        const double need = static_cast<double>(n_q) * left + ITEM_OVERHEAD;
+        const double need = per_tile * left + ITEM_OVERHEAD;
         int take = left;
         if (need > room + slack) {
-          const int can = static_cast<int>(std::floor((room - ITEM_OVERHEAD) / n_q));
+          const int can = static_cast<int>(std::floor((room - ITEM_OVERHEAD - PARTIAL_EXTRA) / per_tile));
           if (can < MIN_PART_TILES) {
             next_cta();
             continue;
@@ -270,8 +278,9 @@ void finalize_schedule(headcast_ctx* c, Schedule& s, std::vector<Proto>& protos,
         w.tile_begin = begin;
         w.tile_end = begin + take;
         parts.push_back(std::make_pair(cta, w));
-        room -= static_cast<double>(n_q) * take + ITEM_OVERHEAD;
-        unassigned -= static_cast<double>(n_q) * take + (begin == 0 ? ITEM_OVERHEAD : 0.0);
+        const bool cut = (take < left) || begin > 0;
+        room -= per_tile * take + ITEM_OVERHEAD + (cut ? PARTIAL_EXTRA : 0.0);
+        unassigned -= per_tile * take + (begin == 0 ? ITEM_OVERHEAD : 0.0);
         begin += take;
         if (room < ITEM_OVERHEAD + MIN_PART_TILES) next_cta();
       }
@@ -429,10 +438,9 @@ int run_schedule(headcast_ctx* c, Schedule& s, const void* q, void* out, bool pr
   p.status = c->status_dev;
   p.trace = nullptr;
   if (c->tracing) {
-    HC_CUDA(c, c->trace_dev.reserve(2 * s.items.size() + 16 * 64));
-    HC_CUDA(c, cudaMemsetAsync(c->trace_dev.ptr, 0, (2 * s.items.size() + 16 * 64) * sizeof(unsigned long long), st));
+    HC_CUDA(c, c->trace_dev.reserve(2 * s.items.size()));
+    HC_CUDA(c, cudaMemsetAsync(c->trace_dev.ptr, 0, 2 * s.items.size() * sizeof(unsigned long long), st));
     p.trace = c->trace_dev.ptr;
-    p.trace_base = static_cast<int32_t>(2 * s.items.size());
     c->trace_items = s.items;
     c->trace_cta_first = s.cta_first;
   }
@@ -603,9 +611,6 @@ int headcast_create(const headcast_config* cfg, headcast_ctx** out) {
     return HC_ERR_UNSUPPORTED;
   }
   c->n_sm = prop.multiProcessorCount;
-#ifdef HC_TIMELINE
-  if (const char* e = getenv("HEADCAST_NUM_CTAS")) c->n_sm = std::max(1, atoi(e));
-#endif
   const size_t mono_bytes = cache_elems(c, c->H) * sizeof(__nv_bfloat16);
   cudaError_t e = cudaSuccess;
   auto step = [&](cudaError_t r) { if (e == cudaSuccess) e = r; };
@@ -993,16 +998,6 @@ int headcast_read_trace(headcast_ctx* c, int64_t* rows_host, int32_t capacity, i
   }
   return HC_OK;
 }
-
-#ifdef HC_TIMELINE
-int headcast_read_timeline(headcast_ctx* c, int64_t* out_host /* [64][16] */) {
-  if (!c || !out_host || c->trace_items.empty()) return HC_ERR_INVALID_ARG;
-  HC_CUDA(c, cudaDeviceSynchronize());
-  HC_CUDA(c, cudaMemcpy(out_host, c->trace_dev.ptr + 2 * c->trace_items.size(), 16 * 64 * sizeof(int64_t),
-                        cudaMemcpyDeviceToHost));
-  return HC_OK;
-}
-#endif
 
 int headcast_check(headcast_ctx* c, void* stream) {
   if (!c) return HC_ERR_INVALID_ARG;

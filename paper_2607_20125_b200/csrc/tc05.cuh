@@ -135,30 +135,81 @@ __host__ __device__ constexpr uint32_t idesc_bf16_f32(uint32_t m, uint32_t n, ui
          ((m >> 4) << 24);
 }
 
-// The same instructions with the descriptors given as (low, high) 32-bit halves and the accumulate flag as a
-// compile-time constant: only the low half (the start address) changes between the k-steps of a tile, so an
-// unrolled issue loop costs one integer add per operand per instruction.
-template <bool ACC>
-__device__ __forceinline__ void mma_ss_lohi(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
-                                            uint32_t idesc) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
-      "setp.ne.b32 p, %6, 0;\n\t"
-      "mov.b64 da, {%1, %2};\n\t"
-      "mov.b64 db, {%3, %4};\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, p;\n\t}"
-      ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "n"(ACC ? 1 : 0)
-      : "memory");
+// Issue blocks.  A tcgen05.mma needs at least ~64 clocks of the tensor pipe whatever its N, and any integer
+// work between two of them (descriptor arithmetic in the issuing thread) costs about as much again.  So the
+// k-steps of one product are issued from ONE asm block whose only other instructions are 64-bit adds on the
+// descriptors' start-address field.
+//
+// S[tmem] = A[smem, K-major] * B[smem, K-major]^T over KSTEPS k-steps of 16; both operands are stored as
+// 64-column blocks of [rows][128 bytes] (128-byte swizzle): k-step kk starts (kk % 4) * 32 bytes into block
+// kk / 4.  a_block16 / b_block16 are the block sizes in units of 16 bytes.
+template <int KSTEPS>
+__device__ __forceinline__ void mma_block_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                             uint32_t a_block16, uint32_t b_block16) {
+  static_assert(KSTEPS == 4 || KSTEPS == 8, "head_dim 64 or 128");
+  if (KSTEPS == 4) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 a, b;\n\t"
+        "setp.ne.b32 p, 0, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t"
+        "setp.eq.b32 p, 0, 0;\n\t"
+        "add.u64 a, %1, 2;\n\tadd.u64 b, %2, 2;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, p;\n\t"
+        "add.u64 a, %1, 4;\n\tadd.u64 b, %2, 4;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, p;\n\t"
+        "add.u64 a, %1, 6;\n\tadd.u64 b, %2, 6;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc)
+        : "memory");
+  } else {
+    const uint64_t a1 = a_desc + a_block16, b1 = b_desc + b_block16;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 a, b;\n\t"
+        "setp.ne.b32 p, 0, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t"
+        "setp.eq.b32 p, 0, 0;\n\t"
+        "add.u64 a, %1, 2;\n\tadd.u64 b, %2, 2;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, p;\n\t"
+        "add.u64 a, %1, 4;\n\tadd.u64 b, %2, 4;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, p;\n\t"
+        "add.u64 a, %1, 6;\n\tadd.u64 b, %2, 6;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, p;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %4, %5, %3, p;\n\t"
+        "add.u64 a, %4, 2;\n\tadd.u64 b, %5, 2;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, p;\n\t"
+        "add.u64 a, %4, 4;\n\tadd.u64 b, %5, 4;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, p;\n\t"
+        "add.u64 a, %4, 6;\n\tadd.u64 b, %5, 6;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "l"(a1), "l"(b1)
+        : "memory");
+  }
 }
-template <bool ACC>
-__device__ __forceinline__ void mma_ts_lohi(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t b_hi,
-                                            uint32_t idesc) {
+
+// O[tmem] (+)= P[tmem, packed bf16, 8 columns per k-step] * V[smem, MN-major] over 8 k-steps of 16 keys;
+// consecutive k-steps of V are 2048 bytes (128 sixteen-byte units) apart.  `accumulate` applies to the first k-step.
+__device__ __forceinline__ void mma_block_ts8(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                              uint32_t accumulate) {
   asm volatile(
-      "{\n\t.reg .pred p;\n\t.reg .b64 db;\n\t"
-      "setp.ne.b32 p, %5, 0;\n\t"
-      "mov.b64 db, {%2, %3};\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n\t}"
-      ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(b_hi), "r"(idesc), "n"(ACC ? 1 : 0)
+      "{\n\t.reg .pred p;\n\t.reg .b64 b;\n\t.reg .b32 a;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t"
+      "setp.eq.b32 p, 0, 0;\n\t"
+      "add.u32 a, %1, 8;\n\tadd.u64 b, %2, 128;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [a], b, %3, p;\n\t"
+      "add.u32 a, %1, 16;\n\tadd.u64 b, %2, 256;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [a], b, %3, p;\n\t"
+      "add.u32 a, %1, 24;\n\tadd.u64 b, %2, 384;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [a], b, %3, p;\n\t"
+      "add.u32 a, %1, 32;\n\tadd.u64 b, %2, 512;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [a], b, %3, p;\n\t"
+      "add.u32 a, %1, 40;\n\tadd.u64 b, %2, 640;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [a], b, %3, p;\n\t"
+      "add.u32 a, %1, 48;\n\tadd.u64 b, %2, 768;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [a], b, %3, p;\n\t"
+      "add.u32 a, %1, 56;\n\tadd.u64 b, %2, 896;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [a], b, %3, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
 
@@ -272,6 +323,28 @@ __device__ __forceinline__ void ex2_pair(float lo, float hi, float& e_lo, float&
   asm("{\n\t.reg .b16 l, u;\n\tmov.b32 {l, u}, %2;\n\tcvt.f32.f16 %0, l;\n\tcvt.f32.f16 %1, u;\n\t}"
       : "=f"(e_lo), "=f"(e_hi)
       : "r"(e));
+}
+
+// 2^x for a packed pair WITHOUT the special-function unit (which can only deliver 16 results per clock per
+// SM, exactly what the tensor pipe consumes at head_dim 128): round x to an integer n with the 1.5 * 2^23
+// trick, evaluate a cubic for 2^(x - n) on [-1/2, 1/2] (relative error 7.5e-5, far below the bf16 rounding of P),
+// and add n to the exponent field.  Inputs must be >= -126 (clamp first); everything runs on the FMA pipe.
+__device__ __forceinline__ void ex2_poly_pair(uint64_t x2, float& e_lo, float& e_hi) {
+  const uint64_t magic = pack_f32x2(12582912.f, 12582912.f), neg_magic = pack_f32x2(-12582912.f, -12582912.f);
+  const uint64_t neg_one = pack_f32x2(-1.f, -1.f);
+  const uint64_t c0 = pack_f32x2(0.9999280572f, 0.9999280572f), c1 = pack_f32x2(0.6932610273f, 0.6932610273f);
+  const uint64_t c2 = pack_f32x2(0.2426111102f, 0.2426111102f), c3 = pack_f32x2(0.0551716015f, 0.0551716015f);
+  const uint64_t t2 = add_f32x2(x2, magic);           // integer part lands in the low mantissa bits
+  const uint64_t r2 = add_f32x2(t2, neg_magic);       // round(x) as a float
+  const uint64_t f2 = fma_f32x2(r2, neg_one, x2);     // x - round(x)
+  uint64_t p2 = fma_f32x2(f2, c3, c2);
+  p2 = fma_f32x2(p2, f2, c1);
+  p2 = fma_f32x2(p2, f2, c0);
+  float t_lo, t_hi, p_lo, p_hi;
+  unpack_f32x2(t2, t_lo, t_hi);
+  unpack_f32x2(p2, p_lo, p_hi);
+  e_lo = __uint_as_float(__float_as_uint(p_lo) + (__float_as_uint(t_lo) << 23));
+  e_hi = __uint_as_float(__float_as_uint(p_hi) + (__float_as_uint(t_hi) << 23));
 }
 
 // 2^lo and 2^hi as packed bf16x2 with ONE special-function operation on bf16 inputs.  The two exponents
