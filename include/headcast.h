@@ -167,6 +167,36 @@ int headcast_check(headcast_ctx* ctx, void* stream);
 
 const char* headcast_last_error(const headcast_ctx* ctx);
 
+/* ---- Dense attention without any allocation -------------------------------------------------------------
+ * (This entry point has no counterpart in the paper; it exists for integration.)
+ *
+ * Some hosts of this library cannot let it allocate device memory: an inference server that has handed the whole
+ * GPU to its own pool (a cudaMalloc from a plug-in then fails, or fragments what the pool believes it owns), or a
+ * frame loop that cannot afford the device-wide synchronisation an allocation or free implies.  For them,
+ * headcast_dense_attend_noalloc computes out[t][h][:] = softmax(scale * q[t][h] . k[:][h]^T) v[:][h] for every head
+ * - the same result as headcast_full_attend on a cache holding k and v - and calls no cudaMalloc, cudaFree or
+ * other allocating routine.  q_dev and out_dev are [n_queries][n_heads][head_dim] bf16, k_dev and v_dev
+ * [n_keys][n_heads][head_dim] bf16, all caller-owned, 16-byte aligned and contiguous.
+ *
+ * The scratch the kernel needs (work list, tensor maps, status word; about 140 KB) is a fixed device array inside
+ * the library: every GPU that loads the library holds it until the process exits.  Consequences:
+ *   - size limit: n_heads * ceil(n_queries / 256) <= HEADCAST_NOALLOC_MAX_ITEMS, head_dim 64 or 128,
+ *     n_heads <= 64; anything larger returns HC_ERR_UNSUPPORTED and does nothing;
+ *   - all calls on one GPU share that array, which keeps the previous call's contents (each call rewrites what
+ *     it uses and clears the status word): two calls whose GPU work overlaps - different streams, or different
+ *     host threads - race on it.  Keep calls on one GPU in one stream, or order them with events;
+ *   - the first call on each device looks up the array's device address and sets the kernel's shared-memory
+ *     attribute (with that device current).  Make that first call before starting any stream capture.
+ * softmax_scale = 0 selects 1/sqrt(head_dim).  Asynchronous on `stream`.  headcast_noalloc_status synchronises
+ * the stream and reports HC_ERR_TIMEOUT if the kernel gave up on a bounded wait; headcast_noalloc_last_error
+ * returns the reason of the last failing call (process-wide buffer). */
+#define HEADCAST_NOALLOC_MAX_ITEMS 2048
+int headcast_dense_attend_noalloc(const void* q_dev, const void* k_dev, const void* v_dev, void* out_dev,
+                                  int32_t n_queries, int32_t n_keys, int32_t n_heads, int32_t head_dim,
+                                  float softmax_scale, void* stream);
+int headcast_noalloc_status(void* stream);
+const char* headcast_noalloc_last_error(void);
+
 #ifdef __cplusplus
 }
 #endif

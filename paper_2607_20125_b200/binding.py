@@ -22,7 +22,8 @@ EXPORTS = ("headcast_default_config", "headcast_create", "headcast_destroy", "he
            "headcast_split_cache", "headcast_attend", "headcast_export_cache", "headcast_n_filled",
            "headcast_launch_count", "headcast_attend_flops", "headcast_check", "headcast_last_error",
            "headcast_set_kernel_timing", "headcast_last_attention_kernel_ms", "headcast_set_tracing",
-           "headcast_read_trace")
+           "headcast_read_trace", "headcast_dense_attend_noalloc", "headcast_noalloc_status",
+           "headcast_noalloc_last_error")
 
 
 class Config(C.Structure):
@@ -73,6 +74,10 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.headcast_last_attention_kernel_ms.argtypes = [vp, f32p]
     lib.headcast_set_tracing.argtypes = [vp, C.c_int32]
     lib.headcast_read_trace.argtypes = [vp, C.POINTER(C.c_int64), C.c_int32, i32p]
+    lib.headcast_dense_attend_noalloc.argtypes = [vp, vp, vp, vp, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_float, vp]
+    lib.headcast_noalloc_status.argtypes = [vp]
+    lib.headcast_noalloc_last_error.argtypes = []
+    lib.headcast_noalloc_last_error.restype = C.c_char_p
     lib.headcast_last_error.argtypes = [vp]
     lib.headcast_last_error.restype = C.c_char_p
     if path is None:
@@ -96,6 +101,28 @@ def _stream() -> int:
 def _ptr(t) -> int:
     assert t.is_cuda and t.is_contiguous(), "tensors handed to the library must be contiguous CUDA tensors"
     return t.data_ptr()
+
+
+def dense_attend_noalloc(q, k, v, out, softmax_scale: float = 0.0) -> None:
+    """Dense attention of q [Lq, H, d] over k, v [Lk, H, d] into out [Lq, H, d] (bf16 CUDA tensors) through the
+    library's allocation-free entry point: for hosts that cannot let the library allocate device memory (a server
+    whose own pool owns the GPU, a loop that cannot take an allocation's device-wide synchronisation).  Calls on
+    one GPU share a fixed scratch array inside the library: keep them on one stream.  Sizes beyond
+    n_heads * ceil(Lq / 256) <= 2048 are rejected."""
+    lib = load_library()
+    n_q, h, d = q.shape
+    rc = lib.headcast_dense_attend_noalloc(_ptr(q), _ptr(k), _ptr(v), _ptr(out), n_q, k.shape[0], h, d,
+                                           float(softmax_scale), _stream())
+    if rc != 0:
+        raise HeadCastError(rc, lib.headcast_noalloc_last_error().decode())
+
+
+def noalloc_status() -> None:
+    """Synchronises the current stream and raises if the allocation-free kernel reported a bounded-wait expiry."""
+    lib = load_library()
+    rc = lib.headcast_noalloc_status(_stream())
+    if rc != 0:
+        raise HeadCastError(rc, lib.headcast_noalloc_last_error().decode())
 
 
 class HeadCast:

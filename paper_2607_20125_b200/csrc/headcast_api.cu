@@ -1007,3 +1007,161 @@ int headcast_check(headcast_ctx* c, void* stream) {
 const char* headcast_last_error(const headcast_ctx* c) { return c ? c->err.c_str() : "null context"; }
 
 }  // extern "C"
+
+// =====================================================================================================
+// Allocation-free dense attention
+// =====================================================================================================
+// Everything the attention kernel needs besides the caller's tensors - the work list, the per-CTA ranges, two
+// tensor maps and the status word - lives in one file-scope device array of fixed size.  Each GPU that loads the
+// library carries these bytes until the process exits.
+namespace {
+
+constexpr int NOALLOC_MAX_ITEMS = HEADCAST_NOALLOC_MAX_ITEMS;
+constexpr int NOALLOC_MAX_CTAS = 1024;
+
+struct NoAllocScratch {
+  CUtensorMap maps[2];                     // K and V of the caller's buffers
+  WorkItem items[NOALLOC_MAX_ITEMS];
+  int32_t cta_first[NOALLOC_MAX_CTAS + 1];
+  int32_t status;
+};
+
+static __device__ __align__(256) unsigned char g_noalloc_scratch[sizeof(NoAllocScratch)];
+
+constexpr int NOALLOC_MAX_DEVICES = 64;
+struct NoAllocDevice {
+  NoAllocScratch* scratch = nullptr;  // device address of g_noalloc_scratch on that GPU
+  int n_sm = 0;
+};
+NoAllocDevice g_noalloc_dev[NOALLOC_MAX_DEVICES];
+
+char g_noalloc_error[256] = "";
+
+int noalloc_fail(int code, const char* msg, cudaError_t e = cudaSuccess) {
+  if (e != cudaSuccess)
+    snprintf(g_noalloc_error, sizeof(g_noalloc_error), "%s: %s", msg, cudaGetErrorString(e));
+  else
+    snprintf(g_noalloc_error, sizeof(g_noalloc_error), "%s", msg);
+  return code;
+}
+
+// Once per device, with that device current: the array's name is only a host-side handle, the kernel needs the
+// address cudaGetSymbolAddress reports for the current device.
+int noalloc_setup(int dev) {
+  NoAllocDevice& d = g_noalloc_dev[dev];
+  if (d.scratch) return HC_OK;
+  cudaDeviceProp prop;
+  cudaError_t e = cudaGetDeviceProperties(&prop, dev);
+  if (e != cudaSuccess) return noalloc_fail(HC_ERR_CUDA, "cudaGetDeviceProperties", e);
+  if (prop.major != 10) return noalloc_fail(HC_ERR_UNSUPPORTED, "this library needs an sm_100 device");
+  void* ptr = nullptr;
+  e = cudaGetSymbolAddress(&ptr, g_noalloc_scratch);
+  if (e != cudaSuccess || !ptr) return noalloc_fail(HC_ERR_CUDA, "cudaGetSymbolAddress(g_noalloc_scratch)", e);
+  e = cudaFuncSetAttribute(attn_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnSmem<128>::DYN_BYTES);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(attn_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnSmem<64>::DYN_BYTES);
+  if (e != cudaSuccess) return noalloc_fail(HC_ERR_CUDA, "cudaFuncSetAttribute", e);
+  d.n_sm = std::min(prop.multiProcessorCount, NOALLOC_MAX_CTAS);
+  d.scratch = static_cast<NoAllocScratch*>(ptr);
+  return HC_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int headcast_dense_attend_noalloc(const void* q, const void* k, const void* v, void* out, int32_t n_queries,
+                                  int32_t n_keys, int32_t n_heads, int32_t head_dim, float softmax_scale, void* stream) {
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out))
+    return noalloc_fail(HC_ERR_INVALID_ARG, "q, k, v and out must be 16-byte aligned device pointers");
+  if (n_queries < 1 || n_keys < 1 || n_heads < 1 || n_heads > MAX_HEADS || (head_dim != 64 && head_dim != 128) ||
+      !(softmax_scale >= 0.f))
+    return noalloc_fail(HC_ERR_INVALID_ARG, "sizes out of range (head_dim 64 or 128, 1..64 heads)");
+  const long long n_items = static_cast<long long>(n_heads) * ((n_queries + 255) / 256);
+  if (n_items > NOALLOC_MAX_ITEMS)
+    return noalloc_fail(HC_ERR_UNSUPPORTED,
+                        "too large for the fixed scratch: n_heads * ceil(n_queries / 256) must not exceed "
+                        "HEADCAST_NOALLOC_MAX_ITEMS");
+  if (static_cast<long long>(n_keys) * n_heads * head_dim >= (1LL << 40) || static_cast<long long>(n_queries) * n_heads >= (1LL << 31))
+    return noalloc_fail(HC_ERR_INVALID_ARG, "sizes out of range");
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return noalloc_fail(HC_ERR_CUDA, "cudaGetDevice", e);
+  if (dev < 0 || dev >= NOALLOC_MAX_DEVICES) return noalloc_fail(HC_ERR_UNSUPPORTED, "device index beyond 63");
+  int rc = noalloc_setup(dev);
+  if (rc != HC_OK) return rc;
+  const NoAllocDevice& d = g_noalloc_dev[dev];
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+
+  // host image of the scratch: thread-local static storage, no heap
+  static thread_local NoAllocScratch host;
+  const uint64_t row_elems = static_cast<uint64_t>(n_heads) * head_dim;
+  if (!make_tmap_bf16_2d(&host.maps[0], k, row_elems, n_keys, row_elems, 128) ||
+      !make_tmap_bf16_2d(&host.maps[1], v, row_elems, n_keys, row_elems, 128))
+    return noalloc_fail(HC_ERR_CUDA, "cuTensorMapEncodeTiled failed or is unavailable");
+  // whole query-tile pairs, dealt round-robin to one CTA per SM (every item has the same key range)
+  const int n_cta = d.n_sm;
+  int n = 0;
+  for (int b = 0; b < n_cta; ++b) {
+    host.cta_first[b] = n;
+    for (long long i = b; i < n_items; i += n_cta) {
+      const int h = static_cast<int>(i % n_heads), q0 = static_cast<int>(i / n_heads) * 256;
+      WorkItem w = range_item(h, 0, h * head_dim, 0, n_keys);
+      w.q_start[0] = q0;
+      w.q_start[1] = q0 + 128;
+      w.q_count[0] = std::min(128, n_queries - q0);
+      w.q_count[1] = std::max(0, std::min(128, n_queries - q0 - 128));
+      w.tile_begin = 0;
+      w.tile_end = w.tiles_per_seg;
+      host.items[n++] = w;
+    }
+  }
+  host.cta_first[n_cta] = n;
+  host.status = 0;  // the array keeps the previous call's contents: the status word must start at zero
+  e = cudaMemcpyAsync(d.scratch->maps, host.maps, sizeof(host.maps), cudaMemcpyHostToDevice, st);
+  if (e == cudaSuccess)
+    e = cudaMemcpyAsync(d.scratch->items, host.items, static_cast<size_t>(n) * sizeof(WorkItem), cudaMemcpyHostToDevice, st);
+  if (e == cudaSuccess)
+    e = cudaMemcpyAsync(d.scratch->cta_first, host.cta_first, (n_cta + 1) * sizeof(int32_t), cudaMemcpyHostToDevice, st);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(&d.scratch->status, &host.status, sizeof(int32_t), cudaMemcpyHostToDevice, st);
+  if (e != cudaSuccess) return noalloc_fail(HC_ERR_CUDA, "copying the work list into the static scratch", e);
+
+  AttnParams p;
+  std::memset(&p, 0, sizeof(p));
+  p.items = d.scratch->items;
+  p.cta_first = d.scratch->cta_first;
+  p.maps = d.scratch->maps;
+  p.q = static_cast<const __nv_bfloat16*>(q);
+  p.out = static_cast<__nv_bfloat16*>(out);
+  p.n_heads = n_heads;
+  p.tokens_per_frame = n_queries;
+  p.grid_w = 1;
+  p.block_tokens = n_queries;
+  const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / std::sqrt(static_cast<float>(head_dim));
+  p.scale_log2e = scale * 1.4426950408889634f;
+  p.status = &d.scratch->status;
+  if (head_dim == 128)
+    attn_kernel<128, false><<<n_cta, ATTN_THREADS, AttnSmem<128>::DYN_BYTES, st>>>(p);
+  else
+    attn_kernel<64, false><<<n_cta, ATTN_THREADS, AttnSmem<64>::DYN_BYTES, st>>>(p);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return noalloc_fail(HC_ERR_CUDA, "launching the attention kernel", e);
+  return HC_OK;
+}
+
+int headcast_noalloc_status(void* stream) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= NOALLOC_MAX_DEVICES || !g_noalloc_dev[dev].scratch)
+    return noalloc_fail(HC_ERR_STATE, "headcast_dense_attend_noalloc has not run on this device");
+  int32_t status = 0;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  cudaError_t e = cudaMemcpyAsync(&status, &g_noalloc_dev[dev].scratch->status, sizeof(status), cudaMemcpyDeviceToHost, st);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  if (e != cudaSuccess) return noalloc_fail(HC_ERR_CUDA, "reading the status word", e);
+  if (status != 0) return noalloc_fail(HC_ERR_TIMEOUT, "the attention kernel gave up on a bounded wait");
+  return HC_OK;
+}
+
+const char* headcast_noalloc_last_error(void) { return g_noalloc_error; }
+
+}  // extern "C"

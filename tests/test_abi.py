@@ -22,7 +22,7 @@ def test_library_exports_every_declared_symbol():
     for n in names:
         assert hasattr(lib, n), n
     for n in names:
-        assert n in binding.EXPORTS or n.endswith("_noalloc"), f"{n} has no binding"
+        assert n in binding.EXPORTS, f"{n} has no binding"
 
 
 def test_default_config_holds_the_papers_constants():
