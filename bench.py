@@ -258,7 +258,7 @@ def main():
     b.synchronize()
     n_sd = sum(1 for v in w.labels if v in (synth.SINK, synth.DUMMY))
     kept_bytes = 2 * 2 * L * D * (n_sd + (H - n_sd) * w.n_blocks)
-    phases["split_ms"] = a.elapsed_time(b)  # includes the allocation of the per-archetype buffers
+    phases["split_ms"] = a.elapsed_time(b)  # one gather launch per cached block
     phases["split_gbs"] = 2 * kept_bytes / phases["split_ms"] / 1e6
 
     n_sink = sum(1 for v in w.labels if v == synth.SINK)
@@ -277,6 +277,16 @@ def main():
     for _ in range(args.warmup):
         step()
     hc.check()
+    # append throughput without launch gaps: 16 launches back to back inside one event pair (1.3 GB at 480P, > L2)
+    flush()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for i in range(16):
+        hc.append(*kv[w.n_blocks + i % n_extra])
+    b.record()
+    b.synchronize()
+    phases["append_split_back_to_back_ms"] = a.elapsed_time(b) / 16
+    phases["append_split_back_to_back_gbs"] = append_bytes / phases["append_split_back_to_back_ms"] / 1e6
     state["i"] = 0
     if dist is not None:
         dist.barrier()

@@ -90,7 +90,8 @@ typedef struct headcast_ctx headcast_ctx;
 /* Fills *cfg with the paper's constants (Sec. 5.1); sizes are left zero for the caller. */
 void headcast_default_config(headcast_config* cfg);
 
-/* Validates cfg, allocates the (zeroed) monolithic cache on the current device and returns a context in *out.
+/* Validates cfg, allocates on the current device the (zeroed) monolithic cache and an equally large zeroed arena
+ * from which headcast_split_cache later carves the per-archetype buffers, and returns a context in *out.
  * Synchronises the device. */
 int headcast_create(const headcast_config* cfg, headcast_ctx** out);
 
@@ -122,7 +123,8 @@ int headcast_get_labels(const headcast_ctx* ctx, int32_t* labels_host);
 
 /* Sec. 4.3: slices the monolithic cache along the head dimension into the Sink-Dummy buffer (one block per
  * head), the Global buffer and the Spatial buffer (full window each).  Needs labels and >= 1 cached block.
- * Allocates the buffers (and frees the monolithic cache unless keep_monolithic).  State becomes SPLIT. */
+ * Allocates nothing (the buffers come from the arena reserved at create); frees the monolithic cache unless
+ * keep_monolithic.  State becomes SPLIT. */
 int headcast_split_cache(headcast_ctx* ctx, void* stream);
 
 /* Sec. 4.4: head-specific attention of one block's queries, one launch for all pathways.  Sink heads read

@@ -5,7 +5,8 @@
 //   - S = Q K^T and O += P V run on tcgen05.mma (M = 128, N = 128 / head_dim, bf16 in, fp32 accumulate)
 //     with S, P and O living in tensor memory (P overlays S as packed bf16 and is fed to the second
 //     product straight from tensor memory);
-//   - K/V tiles (128 keys) arrive through TMA into a 2-stage shared-memory ring (128-byte swizzle);
+//   - K/V tiles (128 keys) arrive through TMA into one 5-slot shared-memory ring (128-byte swizzle), in the
+//     order they are consumed (K0 V0 K1 V1 ...), so loads run two and a half tiles ahead of the products;
 //   - two softmax warpgroups, one per query tile, own one query row per thread (online softmax in the
 //     exp2 domain, a quarter of the exponentials evaluated as a cubic on the FMA pipe to relieve the
 //     special-function unit, rescaling of O only when the running maximum grew by more than 2^8);
@@ -20,6 +21,17 @@
 #include "tc05.cuh"
 
 namespace hc {
+
+// Development aid, compiled out unless HC_TIMELINE is defined: CTA 0 stamps the global timer at the hand-over
+// points of its first 64 key tiles into AttnParams::trace, behind the per-item area (16 slots per tile).
+#ifdef HC_TIMELINE
+#define HC_STAMP(iter, slot)                                                                      \
+  do {                                                                                            \
+    if (p.trace && blockIdx.x == 0 && (iter) < 64) p.trace[p.trace_base + (iter) * 16 + (slot)] = global_timer_ns(); \
+  } while (0)
+#else
+#define HC_STAMP(iter, slot) do { } while (0)
+#endif
 
 struct CellGeom {
   int32_t y0, x0, ch, cw;  // top-left grid position and extent of a deployed Spatial cell
@@ -58,6 +70,7 @@ struct AttnParams {
   int32_t n_heads, tokens_per_frame, grid_w, block_tokens;
   float scale_log2e;       // softmax scale * log2(e)
   int32_t* status;
+  int32_t trace_base;         // HC_TIMELINE only: first timeline slot inside `trace`
   unsigned long long* trace;  // optional [2 * n_items]: globaltimer (ns) when query tile 0's warpgroup starts / ends an item
   // Spatial proxy only
   int32_t radius;
@@ -65,7 +78,7 @@ struct AttnParams {
 };
 
 constexpr int ATTN_THREADS = 384;  // warp 0: TMA, warp 1: MMA, warps 2-3 idle, warps 4-7 / 8-11: softmax for query tile 0 / 1
-constexpr int KV_STAGES = 2;
+constexpr int KV_SLOTS = 5;  // one shared-memory ring for K and V tiles, filled and drained in the order K0 V0 K1 V1 ...
 #ifndef HC_RESCALE_THRESHOLD
 #define HC_RESCALE_THRESHOLD 8.0f
 #endif
@@ -76,9 +89,8 @@ struct AttnSmem {
   static constexpr int BLOCK_BYTES = 128 * 128;      // [128 rows][64 bf16], 128-byte swizzle
   static constexpr int TILE_BYTES = (D / 64) * BLOCK_BYTES;
   static constexpr int Q_OFF = 0;
-  static constexpr int K_OFF = 2 * TILE_BYTES;
-  static constexpr int V_OFF = K_OFF + KV_STAGES * TILE_BYTES;
-  static constexpr int TOTAL = V_OFF + KV_STAGES * TILE_BYTES;
+  static constexpr int KV_OFF = 2 * TILE_BYTES;
+  static constexpr int TOTAL = KV_OFF + KV_SLOTS * TILE_BYTES;
   static constexpr int DYN_BYTES = TOTAL + 1024;  // slack for manual 1024-byte alignment
 };
 
@@ -101,7 +113,7 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const AttnParams 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   __shared__ uint64_t bar_q_full[2], bar_s_full[2], bar_p_full[2], bar_o_full[2];
-  __shared__ uint64_t bar_k_full[KV_STAGES], bar_k_free[KV_STAGES], bar_v_full[KV_STAGES], bar_v_free[KV_STAGES];
+  __shared__ uint64_t bar_kv_full[KV_SLOTS], bar_kv_free[KV_SLOTS];
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag;
 
@@ -113,11 +125,9 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const AttnParams 
       mbar_init(&bar_p_full[t], 128);
       mbar_init(&bar_o_full[t], 1);
     }
-    for (int s = 0; s < KV_STAGES; ++s) {
-      mbar_init(&bar_k_full[s], 1);
-      mbar_init(&bar_k_free[s], 1);
-      mbar_init(&bar_v_full[s], 1);
-      mbar_init(&bar_v_free[s], 1);
+    for (int s = 0; s < KV_SLOTS; ++s) {
+      mbar_init(&bar_kv_full[s], 1);
+      mbar_init(&bar_kv_free[s], 1);
     }
     abort_flag = 0;
     fence_mbar_init();
@@ -146,26 +156,24 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const AttnParams 
         for (int tile = w.tile_begin; tile < w.tile_end; ++tile, ++kt) {
           const int seg = tile / w.tiles_per_seg, c = tile - seg * w.tiles_per_seg;
           const int row = w.kv_row0 + seg * w.seg_stride + c * 128;
-          const uint32_t st = kt % KV_STAGES, ph = (kt / KV_STAGES) & 1;
-          if (!(ok = mbar_wait(&bar_k_free[st], ph ^ 1, abortp, p.status, 11))) break;
-          mbar_arrive_expect_tx(&bar_k_full[st], SM::TILE_BYTES);
-          for (int b = 0; b < NB; ++b)
-            tma_load_2d(smem + SM::K_OFF + st * SM::TILE_BYTES + b * SM::BLOCK_BYTES, kmap, w.kv_x0 + 64 * b, row,
-                        &bar_k_full[st]);
-          if (!(ok = mbar_wait(&bar_v_free[st], ph ^ 1, abortp, p.status, 12))) break;
-          mbar_arrive_expect_tx(&bar_v_full[st], SM::TILE_BYTES);
-          for (int b = 0; b < NB; ++b)
-            tma_load_2d(smem + SM::V_OFF + st * SM::TILE_BYTES + b * SM::BLOCK_BYTES, vmap, w.kv_x0 + 64 * b, row,
-                        &bar_v_full[st]);
+          // ring position g = 2 * kt holds K of this tile, g + 1 its V
+          for (int kv = 0; kv < 2; ++kv) {
+            const uint32_t g = 2 * kt + kv, st = g % KV_SLOTS, ph = (g / KV_SLOTS) & 1;
+            if (!(ok = mbar_wait(&bar_kv_free[st], ph ^ 1, abortp, p.status, 11 + kv))) break;
+            mbar_arrive_expect_tx(&bar_kv_full[st], SM::TILE_BYTES);
+            for (int b = 0; b < NB; ++b)
+              tma_load_2d(smem + SM::KV_OFF + st * SM::TILE_BYTES + b * SM::BLOCK_BYTES, kv ? vmap : kmap,
+                          w.kv_x0 + 64 * b, row, &bar_kv_full[st]);
+          }
+          if (!ok) break;
         }
       }
       if (!ok) {
         // after an expired wait elsewhere: let the copies already in flight land before the CTA leaves
-        for (uint32_t back = 1; back <= KV_STAGES && back <= kt; ++back) {
-          const uint32_t k2 = kt - back, st = k2 % KV_STAGES, ph = (k2 / KV_STAGES) & 1;
+        for (uint32_t back = 1; back <= KV_SLOTS && back <= 2 * kt; ++back) {
+          const uint32_t g = 2 * kt - back, st = g % KV_SLOTS, ph = (g / KV_SLOTS) & 1;
           int local_abort = 0;
-          mbar_wait(&bar_k_full[st], ph, &local_abort, p.status, 13);
-          mbar_wait(&bar_v_full[st], ph, &local_abort, p.status, 13);
+          mbar_wait(&bar_kv_full[st], ph, &local_abort, p.status, 13);
         }
       }
     }
@@ -174,12 +182,11 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const AttnParams 
     if (lane == 0) {
       const uint32_t idesc_s = idesc_bf16_f32(128, 128, 0, 0);
       const uint32_t idesc_o = idesc_bf16_f32(128, D, 0, 1);
-      const uint32_t q_addr = smem_u32(smem + SM::Q_OFF), k_addr = smem_u32(smem + SM::K_OFF),
-                     v_addr = smem_u32(smem + SM::V_OFF);
+      const uint32_t q_addr = smem_u32(smem + SM::Q_OFF), kv_addr = smem_u32(smem + SM::KV_OFF);
       uint32_t kt = 0, q_cnt[2] = {0, 0}, p_cnt[2] = {0, 0};
       bool ok = true;
-      const uint64_t q_desc = smem_desc_sw128(q_addr, 16, 1024), k_desc = smem_desc_sw128(k_addr, 16, 1024);
-      const uint64_t v_desc = smem_desc_sw128(v_addr, SM::BLOCK_BYTES, 1024);
+      const uint64_t q_desc = smem_desc_sw128(q_addr, 16, 1024), k_desc = smem_desc_sw128(kv_addr, 16, 1024);
+      const uint64_t v_desc = smem_desc_sw128(kv_addr, SM::BLOCK_BYTES, 1024);
       auto issue_qk = [&](int t, uint32_t st) {
         mma_block_ss<QK_STEPS>(tmem + S_COL + t * 128, q_desc + ((t * SM::TILE_BYTES) >> 4),
                                k_desc + ((st * SM::TILE_BYTES) >> 4), idesc_s, SM::BLOCK_BYTES >> 4, SM::BLOCK_BYTES >> 4);
@@ -193,8 +200,8 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const AttnParams 
         const int nt = w.tile_end - w.tile_begin;
         const int n_q = w.q_count[1] > 0 ? 2 : 1;
         {
-          const uint32_t st = kt % KV_STAGES, ph = (kt / KV_STAGES) & 1;
-          if (!(ok = mbar_wait(&bar_k_full[st], ph, abortp, p.status, 21))) break;
+          const uint32_t st = (2 * kt) % KV_SLOTS, ph = ((2 * kt) / KV_SLOTS) & 1;
+          if (!(ok = mbar_wait(&bar_kv_full[st], ph, abortp, p.status, 21))) break;
           for (int t = 0; t < n_q && ok; ++t) {
             if (!(ok = mbar_wait(&bar_q_full[t], q_cnt[t] & 1, abortp, p.status, 22))) break;
             ++q_cnt[t];
@@ -203,29 +210,34 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const AttnParams 
             mma_commit(&bar_s_full[t]);
           }
           if (!ok) break;
-          mma_commit(&bar_k_free[st]);
+          mma_commit(&bar_kv_free[st]);
         }
         for (int j = 0; j < nt && ok; ++j) {
-          const uint32_t st = (kt + j) % KV_STAGES, ph = ((kt + j) / KV_STAGES) & 1;
-          const uint32_t st1 = (kt + j + 1) % KV_STAGES, ph1 = ((kt + j + 1) / KV_STAGES) & 1;
-          if (!(ok = mbar_wait(&bar_v_full[st], ph, abortp, p.status, 23))) break;
+          const uint32_t gv = 2 * (kt + j) + 1, gk = gv + 1;  // ring positions of V_j and K_{j+1}
+          const uint32_t st = gv % KV_SLOTS, ph = (gv / KV_SLOTS) & 1;
+          const uint32_t st1 = gk % KV_SLOTS, ph1 = (gk / KV_SLOTS) & 1;
+          if (!(ok = mbar_wait(&bar_kv_full[st], ph, abortp, p.status, 23))) break;
+          HC_STAMP(kt + j, 0);
           for (int t = 0; t < n_q && ok; ++t) {
             if (!(ok = mbar_wait(&bar_p_full[t], p_cnt[t] & 1, abortp, p.status, 24))) break;
+            HC_STAMP(kt + j, 1 + 3 * t);
             ++p_cnt[t];
             tc_fence_after_sync();
             issue_pv(t, st, j > 0);
+            HC_STAMP(kt + j, 2 + 3 * t);
             if (j + 1 < nt) {
-              if (t == 0 && !(ok = mbar_wait(&bar_k_full[st1], ph1, abortp, p.status, 25))) break;
+              if (t == 0 && !(ok = mbar_wait(&bar_kv_full[st1], ph1, abortp, p.status, 25))) break;
               tc_fence_after_sync();
               issue_qk(t, st1);
+              HC_STAMP(kt + j, 3 + 3 * t);
               mma_commit(&bar_s_full[t]);
-              if (t == n_q - 1) mma_commit(&bar_k_free[st1]);
+              if (t == n_q - 1) mma_commit(&bar_kv_free[st1]);
             } else {
               mma_commit(&bar_o_full[t]);
             }
           }
           if (!ok) break;
-          mma_commit(&bar_v_free[st]);
+          mma_commit(&bar_kv_free[st]);
         }
         kt += nt;
       }
@@ -277,6 +289,7 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const AttnParams 
         const int n_valid = min(128, w.seg_len - c * 128);
         const int tok0 = PROXY ? (w.kv_row0 + c * 128) : 0;  // in-frame token of this tile's first key
         if (!(ok = mbar_wait(&bar_s_full[t], s_cnt & 1, abortp, p.status, 31))) break;
+        if (r == 0) HC_STAMP(s_cnt, 7 + 4 * t);
         ++s_cnt;
         tc_fence_after_sync();
         // the whole logit row of this thread: 128 fp32 values, loaded with four back-to-back TMEM reads
@@ -284,6 +297,7 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const AttnParams 
 #pragma unroll
         for (int ch = 0; ch < 4; ++ch) tmem_ld32(s_addr + ch * 32, reinterpret_cast<uint32_t(&)[32]>(sv[ch * 32]));
         tmem_wait_ld();
+        if (r == 0) HC_STAMP(s_cnt - 1, 8 + 4 * t);
         // keys this row must not see get a logit of -inf: the ragged tail of a segment, and for the
         // Spatial proxy every key outside the (2r+1)^2 neighbourhood of the query's grid position
         if (PROXY) {
@@ -330,6 +344,7 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const AttnParams 
           }
         }
         const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
+        if (r == 0) HC_STAMP(s_cnt - 1, 9 + 4 * t);
         // p = 2^(s * c - m) for two keys per special-function operation, row sum in fp32, bf16 pack into the
         // first 64 columns of S_t
         const uint64_t c2 = pack_f32x2(p.scale_log2e, p.scale_log2e), m2 = pack_f32x2(-m_use, -m_use);
@@ -366,6 +381,7 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const AttnParams 
         tmem_wait_st();
         tc_fence_before_sync();
         mbar_arrive(&bar_p_full[t]);
+        if (r == 0) HC_STAMP(s_cnt - 1, 10 + 4 * t);
       }
       if (!ok) break;
       // ---- epilogue

@@ -80,6 +80,7 @@ struct headcast_ctx {
   std::vector<int> cell_tok_off;  // tokens per frame in earlier cells
 
   __nv_bfloat16 *mono_k = nullptr, *mono_v = nullptr;
+  __nv_bfloat16 *arena_k = nullptr, *arena_v = nullptr;  // zeroed at create; the per-archetype buffers are carved from it
   __nv_bfloat16 *sd_k = nullptr, *sd_v = nullptr, *g_k = nullptr, *g_v = nullptr, *sp_k = nullptr, *sp_v = nullptr;
   int32_t *sp_base = nullptr, *sp_nc = nullptr;
   CellGeom* cells_dev = nullptr;
@@ -215,10 +216,10 @@ WorkItem range_item(int head, int map, int x0, long long row0, int n_keys) {
 }
 
 // Cost model of the scheduler, in units of the time one key tile takes with both query tiles in flight
-// (fitted to per-item timings from headcast_read_trace on B200): a lone query tile still needs 0.8 of that
+// (fitted to per-item timings from headcast_read_trace on B200): a lone query tile still needs 0.86 of that
 // because the chain S -> softmax -> P -> next S is latency bound; every item pays for its query load, pipeline
 // fill and epilogue; a partial result costs an extra round trip through global memory.
-constexpr double TILE_COST_PAIR = 1.0, TILE_COST_SINGLE = 0.8;
+constexpr double TILE_COST_PAIR = 1.0, TILE_COST_SINGLE = 0.86;
 constexpr double ITEM_OVERHEAD = 3.5;
 constexpr double PARTIAL_EXTRA = 1.0;
 constexpr int MIN_PART_TILES = 4;  // never cut a key range into pieces shorter than this
@@ -438,9 +439,11 @@ int run_schedule(headcast_ctx* c, Schedule& s, const void* q, void* out, bool pr
   p.status = c->status_dev;
   p.trace = nullptr;
   if (c->tracing) {
-    HC_CUDA(c, c->trace_dev.reserve(2 * s.items.size()));
-    HC_CUDA(c, cudaMemsetAsync(c->trace_dev.ptr, 0, 2 * s.items.size() * sizeof(unsigned long long), st));
+    const size_t trace_words = 2 * s.items.size() + 16 * 64;  // per-item stamps, then the HC_TIMELINE area
+    HC_CUDA(c, c->trace_dev.reserve(trace_words));
+    HC_CUDA(c, cudaMemsetAsync(c->trace_dev.ptr, 0, trace_words * sizeof(unsigned long long), st));
     p.trace = c->trace_dev.ptr;
+    p.trace_base = static_cast<int32_t>(2 * s.items.size());
     c->trace_items = s.items;
     c->trace_cta_first = s.cta_first;
   }
@@ -616,6 +619,8 @@ int headcast_create(const headcast_config* cfg, headcast_ctx** out) {
   auto step = [&](cudaError_t r) { if (e == cudaSuccess) e = r; };
   step(cudaMalloc(&c->mono_k, mono_bytes));
   step(cudaMalloc(&c->mono_v, mono_bytes));
+  step(cudaMalloc(&c->arena_k, mono_bytes));
+  step(cudaMalloc(&c->arena_v, mono_bytes));
   step(cudaMalloc(&c->sp_base, c->T_f * sizeof(int32_t)));
   step(cudaMalloc(&c->sp_nc, c->T_f * sizeof(int32_t)));
   step(cudaMalloc(&c->cells_dev, c->cells.size() * sizeof(CellGeom)));
@@ -624,6 +629,8 @@ int headcast_create(const headcast_config* cfg, headcast_ctx** out) {
   if (e == cudaSuccess) {
     step(cudaMemset(c->mono_k, 0, mono_bytes));
     step(cudaMemset(c->mono_v, 0, mono_bytes));
+    step(cudaMemset(c->arena_k, 0, mono_bytes));
+    step(cudaMemset(c->arena_v, 0, mono_bytes));
     step(cudaMemset(c->status_dev, 0, sizeof(int32_t)));
     step(cudaMemcpy(c->sp_base, sp_base.data(), c->T_f * sizeof(int32_t), cudaMemcpyHostToDevice));
     step(cudaMemcpy(c->sp_nc, sp_nc.data(), c->T_f * sizeof(int32_t), cudaMemcpyHostToDevice));
@@ -644,8 +651,7 @@ int headcast_create(const headcast_config* cfg, headcast_ctx** out) {
 int headcast_destroy(headcast_ctx* c) {
   if (!c) return HC_OK;
   cudaDeviceSynchronize();
-  void* ptrs[] = {c->mono_k, c->mono_v, c->sd_k, c->sd_v, c->g_k, c->g_v, c->sp_k, c->sp_v,
-                  c->sp_base, c->sp_nc, c->cells_dev, c->maps_dev, c->status_dev};
+  void* ptrs[] = {c->mono_k, c->mono_v, c->arena_k, c->arena_v, c->sp_base, c->sp_nc, c->cells_dev, c->maps_dev, c->status_dev};
   for (void* p : ptrs)
     if (p) cudaFree(p);
   if (c->ev_a) cudaEventDestroy(c->ev_a);
@@ -834,24 +840,17 @@ int headcast_split_cache(headcast_ctx* c, void* stream) {
   if (c->slots.empty()) return fail(c, HC_ERR_STATE, "the cache is empty");
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   assign_classes(c);
-  const size_t esz = sizeof(__nv_bfloat16);
+  // carve the three buffers out of the arena reserved (and zeroed) at create: no allocation on this path
   const int n_sd = c->n_cls[CLS_SINK] + c->n_cls[CLS_DUMMY];
-  const size_t sd_bytes = static_cast<size_t>(n_sd) * c->L * c->D * esz;
-  const size_t g_bytes = cache_elems(c, c->n_cls[CLS_GLOBAL]) * esz;
-  const size_t sp_bytes = cache_elems(c, c->n_cls[CLS_SPATIAL]) * esz;
-  struct { __nv_bfloat16** p; size_t bytes; } bufs[] = {{&c->sd_k, sd_bytes}, {&c->sd_v, sd_bytes}, {&c->g_k, g_bytes},
-                                                        {&c->g_v, g_bytes},   {&c->sp_k, sp_bytes}, {&c->sp_v, sp_bytes}};
-  for (auto& b : bufs) {
-    if (b.bytes == 0) continue;
-    cudaError_t e = cudaMalloc(b.p, b.bytes);
-    if (e == cudaSuccess) e = cudaMemsetAsync(*b.p, 0, b.bytes, st);
-    if (e != cudaSuccess) {
-      for (auto& f : bufs)
-        if (*f.p) { cudaFree(*f.p); *f.p = nullptr; }
-      return fail(c, e == cudaErrorMemoryAllocation ? HC_ERR_NOMEM : HC_ERR_CUDA, "allocating the per-archetype buffers: %s",
-                  cudaGetErrorString(e));
-    }
-  }
+  const size_t sd_elems = static_cast<size_t>(n_sd) * c->L * c->D;
+  const size_t g_elems = cache_elems(c, c->n_cls[CLS_GLOBAL]);
+  const size_t sp_elems = cache_elems(c, c->n_cls[CLS_SPATIAL]);
+  c->sd_k = sd_elems ? c->arena_k : nullptr;
+  c->sd_v = sd_elems ? c->arena_v : nullptr;
+  c->g_k = g_elems ? c->arena_k + sd_elems : nullptr;
+  c->g_v = g_elems ? c->arena_v + sd_elems : nullptr;
+  c->sp_k = sp_elems ? c->arena_k + sd_elems + g_elems : nullptr;
+  c->sp_v = sp_elems ? c->arena_v + sd_elems + g_elems : nullptr;
   const size_t block_elems = static_cast<size_t>(c->L) * c->H * c->D;
   for (size_t i = 0; i < c->slots.size(); ++i) {
     RouteParams r;
@@ -998,6 +997,16 @@ int headcast_read_trace(headcast_ctx* c, int64_t* rows_host, int32_t capacity, i
   }
   return HC_OK;
 }
+
+#ifdef HC_TIMELINE
+int headcast_read_timeline(headcast_ctx* c, int64_t* out_host /* [64][16] */) {
+  if (!c || !out_host || c->trace_items.empty()) return HC_ERR_INVALID_ARG;
+  HC_CUDA(c, cudaDeviceSynchronize());
+  HC_CUDA(c, cudaMemcpy(out_host, c->trace_dev.ptr + 2 * c->trace_items.size(), 16 * 64 * sizeof(int64_t),
+                        cudaMemcpyDeviceToHost));
+  return HC_OK;
+}
+#endif
 
 int headcast_check(headcast_ctx* c, void* stream) {
   if (!c) return HC_ERR_INVALID_ARG;
