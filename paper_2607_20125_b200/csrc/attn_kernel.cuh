@@ -5,9 +5,9 @@
 //   - S = Q K^T and O += P V run on tcgen05.mma (M = 128, N = 128 / head_dim, bf16 in, fp32 accumulate)
 //     with S, P and O living in tensor memory (P overlays S as packed bf16 and is fed to the second
 //     product straight from tensor memory);
-//   - K/V tiles (128 keys) arrive through TMA into one 5-slot shared-memory ring (128-byte swizzle), in the
-//     order they are consumed (K0 V0 K1 V1 ...), so loads run two and a half tiles ahead of the products;
-//   - two softmax warpgroups, one per query tile, own one query row per thread (online softmax in the
+//   - K/V tiles (128 keys) arrive through TMA into one 4-slot shared-memory ring (128-byte swizzle), in the
+//     order they are consumed (K0 V0 K1 V1 ...), so loads run two tiles ahead of the products;
+//   - sixteen softmax warps, eight per query tile, two threads per query row (online softmax in the
 //     exp2 domain, a quarter of the exponentials evaluated as a cubic on the FMA pipe to relieve the
 //     special-function unit, rescaling of O only when the running maximum grew by more than 2^8);
 //   - warp 0 is the TMA producer, warp 1 issues every MMA.
@@ -77,8 +77,12 @@ struct AttnParams {
   int32_t mid_seg_lo, mid_seg_hi, last_seg_lo, last_seg_hi;  // segments (cached frames) of the middle / newest blocks
 };
 
-constexpr int ATTN_THREADS = 384;  // warp 0: TMA, warp 1: MMA, warps 2-3 idle, warps 4-7 / 8-11: softmax for query tile 0 / 1
-constexpr int KV_SLOTS = 5;  // one shared-memory ring for K and V tiles, filled and drained in the order K0 V0 K1 V1 ...
+constexpr int ATTN_THREADS = 576;  // warp 0: TMA, warp 1: MMA, warps 2-9 / 10-17: softmax for query tile 0 / 1 (112 registers each)
+constexpr int SOFTMAX_WARPS = 8;    // per query tile: two threads per row, each owning 64 of the tile's 128 keys
+constexpr int KV_SLOTS = 4;  // one shared-memory ring for K and V tiles, filled and drained in the order K0 V0 K1 V1 ...
+#ifndef HC_POLY_MASK
+#define HC_POLY_MASK 3  // pairs whose index has all these bits set take the polynomial exponential (3: every 4th)
+#endif
 #ifndef HC_RESCALE_THRESHOLD
 #define HC_RESCALE_THRESHOLD 8.0f
 #endif
@@ -102,6 +106,26 @@ __device__ __forceinline__ int cell_query_token(const CellGeom& g, int p, int to
   return f * tokens_per_frame + (g.y0 + dy) * grid_w + g.x0 + dx;
 }
 
+// Sets the logits of keys a query row must not see to -inf: columns >= n_valid (ragged tail of a segment) and,
+// for the Spatial proxy, keys outside the (2r+1)^2 neighbourhood of the query's grid position (qy, qx); tok0 is
+// the in-frame token index of column 0.
+template <bool PROXY>
+__device__ __forceinline__ void mask_logits(uint32_t (&sv)[32], int n_valid, int tok0, int qy, int qx, int radius, int grid_w) {
+  if (PROXY) {
+    int ky = tok0 / grid_w, kx = tok0 - ky * grid_w;
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+      const bool a = (i < n_valid) && (abs(ky - qy) <= radius) && (abs(kx - qx) <= radius);
+      if (!a) sv[i] = 0xff800000u;
+      if (++kx == grid_w) { kx = 0; ++ky; }
+    }
+  } else if (n_valid < 32) {
+#pragma unroll
+    for (int i = 0; i < 32; ++i)
+      if (i >= n_valid) sv[i] = 0xff800000u;
+  }
+}
+
 template <int D, bool PROXY>
 __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const AttnParams p) {
   using SM = AttnSmem<D>;
@@ -112,7 +136,8 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const AttnParams 
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  __shared__ uint64_t bar_q_full[2], bar_s_full[2], bar_p_full[2], bar_o_full[2];
+  __shared__ uint64_t bar_q_full[2], bar_s_full[2], bar_p_full[2], bar_o_full[2], bar_pair[2];
+  __shared__ float pair_val[2][2][2][128];  // [query tile][parity][column half][row]: values the two threads of a row swap
   __shared__ uint64_t bar_kv_full[KV_SLOTS], bar_kv_free[KV_SLOTS];
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag;
@@ -120,10 +145,13 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const AttnParams 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   if (tid == 0) {
     for (int t = 0; t < 2; ++t) {
-      mbar_init(&bar_q_full[t], 128);
+      // softmax warps arrive once per warp (lane 0, after __syncwarp): 256 arrivals on one mbarrier would be
+      // 256 serialised shared-memory atomics per tile
+      mbar_init(&bar_q_full[t], SOFTMAX_WARPS);
       mbar_init(&bar_s_full[t], 1);
-      mbar_init(&bar_p_full[t], 128);
+      mbar_init(&bar_p_full[t], SOFTMAX_WARPS);
       mbar_init(&bar_o_full[t], 1);
+      mbar_init(&bar_pair[t], SOFTMAX_WARPS);
     }
     for (int s = 0; s < KV_SLOTS; ++s) {
       mbar_init(&bar_kv_full[s], 1);
@@ -143,6 +171,7 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const AttnParams 
   volatile int* abortp = &abort_flag;
 
   const int item_lo = p.cta_first[blockIdx.x], item_hi = p.cta_first[blockIdx.x + 1];
+
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
@@ -242,38 +271,58 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const AttnParams 
         kt += nt;
       }
     }
-  } else if (warp >= 4) {
-    // ------------------------------------------------------------------ softmax + epilogue warpgroups
-    const int t = (warp - 4) >> 2;                  // query tile of this warpgroup
+  } else {
+    // ------------------------------------------------------------------ softmax + epilogue warps
+    // Eight warps per query tile.  A warp may only touch the 32 TMEM lanes (rows) of its warp-id quarter, and a
+    // lone warp cannot issue fast enough to keep up with the tensor pipe, so every row is shared by two threads
+    // of two warps on the same scheduler: each owns 64 of the tile's 128 keys (and half of the output columns)
+    // and they swap their row maxima through shared memory once per tile.
+    const int t = (warp - 2) >> 3;                  // query tile
+    const int half = ((warp - 2) >> 2) & 1;         // which 64 keys / which half of the output columns
     const int r = ((warp & 3) << 5) | lane;         // row inside the tile == TMEM lane
     const uint32_t lane_off = static_cast<uint32_t>((warp & 3) << 5) << 16;
-    const uint32_t s_addr = tmem + lane_off + S_COL + t * 128;
-    const uint32_t o_addr = tmem + lane_off + O_COL + t * 128;
+    const uint32_t s_addr = tmem + lane_off + S_COL + t * 128 + half * 64;   // this thread's logits
+    const uint32_t p_addr = s_addr;  // its share of P (packed bf16) goes over the first 32 columns of its own logits
+    constexpr int OC = D / 2;                                                // output columns per thread
+    const uint32_t o_addr = tmem + lane_off + O_COL + t * 128 + half * OC;
     uint8_t* sq = smem + SM::Q_OFF + t * SM::TILE_BYTES;
-    uint32_t s_cnt = 0, o_cnt = 0;
+    uint32_t s_cnt = 0, o_cnt = 0, x_cnt = 0;
     bool ok = true;
+    // swaps one float with the other thread of the row (bounded wait like every other wait here)
+    auto swap_with_partner = [&](float mine, float& theirs) -> bool {
+      const int par = x_cnt & 1;
+      pair_val[t][par][half][r] = mine;
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&bar_pair[t]);
+      if (!mbar_wait(&bar_pair[t], par, abortp, p.status, 34)) return false;
+      ++x_cnt;
+      theirs = pair_val[t][par][half ^ 1][r];
+      return true;
+    };
     for (int it = item_lo; it < item_hi && ok; ++it) {
       const WorkItem w = p.items[it];
       if (w.q_count[t] == 0) continue;
-      if (p.trace && t == 0 && r == 0) p.trace[2 * it] = global_timer_ns();
+      if (p.trace && t == 0 && r == 0 && half == 0) p.trace[2 * it] = global_timer_ns();
       const bool row_valid = r < w.q_count[t];
       int token = 0;
       if (row_valid) {
         token = w.q_start[t] + r;
         if (w.cell >= 0) token = cell_query_token(p.cells[w.cell], token, p.tokens_per_frame, p.grid_w);
       }
-      // ---- stage this thread's query row into shared memory (swizzled); invalid rows are zero
+      // ---- stage this thread's half of its query row into shared memory (swizzled); invalid rows are zero
       {
         const uint4* src = reinterpret_cast<const uint4*>(p.q + (static_cast<size_t>(token) * p.n_heads + w.head) * D);
 #pragma unroll
-        for (int c = 0; c < D / 8; ++c) {
+        for (int cc = 0; cc < D / 16; ++cc) {
+          const int c = half * (D / 16) + cc;
           uint4 v = make_uint4(0, 0, 0, 0);
           if (row_valid) v = __ldg(src + c);
           *reinterpret_cast<uint4*>(sq + (c / 8) * SM::BLOCK_BYTES + sw128_offset(r, c % 8)) = v;
         }
         fence_proxy_async_smem();
         tc_fence_before_sync();  // orders this thread's TMEM reads of the previous item before the arrive
-        mbar_arrive(&bar_q_full[t]);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&bar_q_full[t]);
       }
       int qy = 0, qx = 0;
       if (PROXY) {
@@ -281,49 +330,46 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const AttnParams 
         qy = pos / p.grid_w;
         qx = pos - qy * p.grid_w;
       }
-      float m_ref = -INFINITY, l_sum = 0.f, l_mid = 0.f;
+      float m_ref = -INFINITY, l_sum = 0.f, l_mid = 0.f;  // l_* cover this thread's 64 keys per tile only
       const int nt = w.tile_end - w.tile_begin;
       for (int j = 0; j < nt; ++j) {
         const int tile = w.tile_begin + j;
         const int seg = tile / w.tiles_per_seg, c = tile - seg * w.tiles_per_seg;
-        const int n_valid = min(128, w.seg_len - c * 128);
-        const int tok0 = PROXY ? (w.kv_row0 + c * 128) : 0;  // in-frame token of this tile's first key
+        const int n_valid = min(128, w.seg_len - c * 128) - half * 64;  // valid keys among this thread's 64
+        const int tok0 = PROXY ? (w.kv_row0 + c * 128 + half * 64) : 0;  // in-frame token of its first key
         if (!(ok = mbar_wait(&bar_s_full[t], s_cnt & 1, abortp, p.status, 31))) break;
-        if (r == 0) HC_STAMP(s_cnt, 7 + 4 * t);
+        if (r == 0 && half == 0) HC_STAMP(s_cnt, 7 + 4 * t);
         ++s_cnt;
         tc_fence_after_sync();
-        // the whole logit row of this thread: 128 fp32 values, loaded with four back-to-back TMEM reads
-        uint32_t sv[128];
+        // pass 1: maximum of this thread's 64 logits (32 columns at a time; they are read again in pass 2, which
+        // keeps the live registers low enough for 576 threads per CTA).  Keys this row must not see count as -inf:
+        // the ragged tail of a segment, and for the Spatial proxy every key outside the (2r+1)^2 neighbourhood.
+        float mx;
+        {
+          float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-        for (int ch = 0; ch < 4; ++ch) tmem_ld32(s_addr + ch * 32, reinterpret_cast<uint32_t(&)[32]>(sv[ch * 32]));
-        tmem_wait_ld();
-        if (r == 0) HC_STAMP(s_cnt - 1, 8 + 4 * t);
-        // keys this row must not see get a logit of -inf: the ragged tail of a segment, and for the
-        // Spatial proxy every key outside the (2r+1)^2 neighbourhood of the query's grid position
-        if (PROXY) {
-          int ky = tok0 / p.grid_w, kx = tok0 - ky * p.grid_w;
+          for (int ch = 0; ch < 2; ++ch) {
+            uint32_t sv[32];
+            tmem_ld32(s_addr + ch * 32, sv);
+            tmem_wait_ld();
+            mask_logits<PROXY>(sv, n_valid - ch * 32, tok0 + ch * 32, qy, qx, p.radius, p.grid_w);
 #pragma unroll
-          for (int i = 0; i < 128; ++i) {
-            const bool a = (i < n_valid) && (abs(ky - qy) <= p.radius) && (abs(kx - qx) <= p.radius);
-            if (!a) sv[i] = 0xff800000u;
-            if (++kx == p.grid_w) { kx = 0; ++ky; }
+            for (int i = 0; i < 32; i += 8) {
+              mx4[0] = max3(mx4[0], __uint_as_float(sv[i]), __uint_as_float(sv[i + 1]));
+              mx4[1] = max3(mx4[1], __uint_as_float(sv[i + 2]), __uint_as_float(sv[i + 3]));
+              mx4[2] = max3(mx4[2], __uint_as_float(sv[i + 4]), __uint_as_float(sv[i + 5]));
+              mx4[3] = max3(mx4[3], __uint_as_float(sv[i + 6]), __uint_as_float(sv[i + 7]));
+            }
           }
-        } else if (n_valid < 128) {
-#pragma unroll
-          for (int i = 0; i < 128; ++i)
-            if (i >= n_valid) sv[i] = 0xff800000u;
+          mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
         }
-        float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-#pragma unroll
-        for (int i = 0; i < 128; i += 8) {
-          mx4[0] = max3(mx4[0], __uint_as_float(sv[i]), __uint_as_float(sv[i + 1]));
-          mx4[1] = max3(mx4[1], __uint_as_float(sv[i + 2]), __uint_as_float(sv[i + 3]));
-          mx4[2] = max3(mx4[2], __uint_as_float(sv[i + 4]), __uint_as_float(sv[i + 5]));
-          mx4[3] = max3(mx4[3], __uint_as_float(sv[i + 6]), __uint_as_float(sv[i + 7]));
-        }
-        float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
-        mx *= p.scale_log2e;  // scale > 0, so the maximum commutes with it
-        // running maximum: move the reference only when some row of the warp outgrew it by 2^8
+        if (r == 0 && half == 0) HC_STAMP(s_cnt - 1, 8 + 4 * t);
+        float mx_other;
+        if (!(ok = swap_with_partner(mx, mx_other))) break;
+        mx = fmaxf(mx, mx_other) * p.scale_log2e;  // row maximum; scale > 0, so the maximum commutes with it
+        if (r == 0 && half == 0) HC_STAMP(s_cnt - 1, 9 + 4 * t);
+        // running maximum: move the reference only when some row of the warp outgrew it by 2^8.  Both threads of
+        // a row see the same maximum and sit in the same lane of their warps, so both warps decide alike.
         const bool grow = mx > m_ref + RESCALE_THRESHOLD || (m_ref == -INFINITY && mx > -INFINITY);
         if (__any_sync(0xffffffffu, grow)) {
           const float m_new = fmaxf(m_ref, mx);
@@ -331,9 +377,9 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const AttnParams 
           l_sum *= alpha;
           l_mid *= alpha;
           m_ref = m_new;
-          if (j > 0) {  // O_t holds the products of the earlier tiles: bring them to the new reference
+          if (j > 0) {  // O_t holds the products of the earlier tiles: bring this thread's columns to the new reference
 #pragma unroll 1
-            for (int ch = 0; ch < D / 32; ++ch) {
+            for (int ch = 0; ch < OC / 32; ++ch) {
               uint32_t v[32];
               tmem_ld32(o_addr + ch * 32, v);
               tmem_wait_ld();
@@ -344,21 +390,22 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const AttnParams 
           }
         }
         const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
-        if (r == 0) HC_STAMP(s_cnt - 1, 9 + 4 * t);
-        // p = 2^(s * c - m) for two keys per special-function operation, row sum in fp32, bf16 pack into the
-        // first 64 columns of S_t
+        // pass 2: p = 2^(s * c - m), row sum in fp32, bf16 pack over the first 32 columns of this thread's logits
         const uint64_t c2 = pack_f32x2(p.scale_log2e, p.scale_log2e), m2 = pack_f32x2(-m_use, -m_use);
         uint64_t sum2[2] = {0ull, 0ull};
 #pragma unroll
-        for (int ch = 0; ch < 4; ++ch) {
+        for (int ch = 0; ch < 2; ++ch) {
+          uint32_t sv[32];
+          tmem_ld32(s_addr + ch * 32, sv);
+          tmem_wait_ld();
+          mask_logits<PROXY>(sv, n_valid - ch * 32, tok0 + ch * 32, qy, qx, p.radius, p.grid_w);
           uint32_t pk[16];
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
-            const uint64_t x2 = fma_f32x2(
-                pack_f32x2(__uint_as_float(sv[ch * 32 + 2 * i]), __uint_as_float(sv[ch * 32 + 2 * i + 1])), c2, m2);
+            const uint64_t x2 = fma_f32x2(pack_f32x2(__uint_as_float(sv[2 * i]), __uint_as_float(sv[2 * i + 1])), c2, m2);
             float x0, x1, e0, e1;
             unpack_f32x2(x2, x0, x1);
-            if ((i & 3) == 3) {
+            if ((i & HC_POLY_MASK) == HC_POLY_MASK) {
               // every fourth pair takes the polynomial route on the FMA pipe: the special-function unit alone
               // cannot produce 128 x 128 exponentials in the time the tensor pipe needs for the tile
               ex2_poly_pair(pack_f32x2(fmaxf(x0, -126.f), fmaxf(x1, -126.f)), e0, e1);
@@ -369,7 +416,7 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const AttnParams 
             pk[i] = pack_bf16x2(e0, e1);
             sum2[i & 1] = add_f32x2(sum2[i & 1], pack_f32x2(e0, e1));
           }
-          tmem_st16(s_addr + ch * 16, pk);
+          tmem_st16(p_addr + ch * 16, pk);
         }
         float t0, t1, t2, t3;
         unpack_f32x2(sum2[0], t0, t1);
@@ -380,19 +427,27 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const AttnParams 
           l_mid += tile_sum;
         tmem_wait_st();
         tc_fence_before_sync();
-        mbar_arrive(&bar_p_full[t]);
-        if (r == 0) HC_STAMP(s_cnt - 1, 10 + 4 * t);
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&bar_p_full[t]);
+        if (r == 0 && half == 0) HC_STAMP(s_cnt - 1, 10 + 4 * t);
       }
       if (!ok) break;
-      // ---- epilogue
+      // ---- epilogue: row sums of the two halves are added, each thread normalises and stores its output columns
+      float other;
+      if (!(ok = swap_with_partner(l_sum, other))) break;
+      l_sum += other;
+      if (PROXY) {
+        if (!(ok = swap_with_partner(l_mid, other))) break;
+        l_mid += other;
+      }
       if (!(ok = mbar_wait(&bar_o_full[t], o_cnt & 1, abortp, p.status, 32))) break;
       ++o_cnt;
       tc_fence_after_sync();
       const float inv = (l_sum > 0.f) ? 1.f / l_sum : 0.f;
       const float mult = (w.out_mode == OUT_PARTIAL) ? 1.f : inv;
-      const size_t row_elem = (static_cast<size_t>(token) * p.n_heads + w.head) * D;
+      const size_t row_elem = (static_cast<size_t>(token) * p.n_heads + w.head) * D + half * OC;
 #pragma unroll 1
-      for (int ch = 0; ch < D / 32; ++ch) {
+      for (int ch = 0; ch < OC / 32; ++ch) {
         uint32_t v[32];
         tmem_ld32(o_addr + ch * 32, v);
         tmem_wait_ld();
@@ -410,7 +465,7 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const AttnParams 
           }
         } else {
           float* base = (w.out_mode == OUT_PARTIAL)
-                            ? p.part_o + (static_cast<size_t>(w.out_slot) * 256 + t * 128 + r) * D
+                            ? p.part_o + (static_cast<size_t>(w.out_slot) * 256 + t * 128 + r) * D + half * OC
                             : p.f32_o + static_cast<size_t>(w.out_slot) * p.block_tokens * p.n_heads * D + row_elem;
           float4* dst = reinterpret_cast<float4*>(base + ch * 32);
 #pragma unroll
@@ -419,7 +474,7 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const AttnParams 
                                  __uint_as_float(v[4 * i + 2]) * mult, __uint_as_float(v[4 * i + 3]) * mult);
         }
       }
-      if (row_valid) {
+      if (row_valid && half == 0) {
         if (w.out_mode == OUT_PARTIAL) {
           p.part_ml[static_cast<size_t>(w.out_slot) * 256 + t * 128 + r] = make_float2(m_ref, l_sum);
         } else if (w.out_mode == OUT_F32_LSE) {
@@ -430,7 +485,7 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const AttnParams 
           if (PROXY) p.f32_lse[(w.out_slot + 1) * lh + idx] = (l_mid > 0.f) ? m_ref * ln2 + __logf(l_mid) : -INFINITY;
         }
       }
-      if (p.trace && t == 0 && r == 0) p.trace[2 * it + 1] = global_timer_ns();
+      if (p.trace && t == 0 && r == 0 && half == 0) p.trace[2 * it + 1] = global_timer_ns();
     }
   }
   // ------------------------------------------------------------------ teardown

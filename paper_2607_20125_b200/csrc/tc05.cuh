@@ -187,7 +187,9 @@ __device__ __forceinline__ void mma_block_ss(uint32_t d_tmem, uint64_t a_desc, u
 }
 
 // O[tmem] (+)= P[tmem, packed bf16, 8 columns per k-step] * V[smem, MN-major] over 8 k-steps of 16 keys;
-// consecutive k-steps of V are 2048 bytes (128 sixteen-byte units) apart.  `accumulate` applies to the first k-step.
+// consecutive k-steps of V are 2048 bytes (128 sixteen-byte units) apart.  P is stored in two pieces: keys 0..63
+// in columns a .. a+31, keys 64..127 in columns a+64 .. a+95 (each piece over the logits it was computed from).
+// `accumulate` applies to the first k-step.
 __device__ __forceinline__ void mma_block_ts8(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
                                               uint32_t accumulate) {
   asm volatile(
@@ -201,13 +203,13 @@ __device__ __forceinline__ void mma_block_ts8(uint32_t d_tmem, uint32_t a_tmem, 
       "tcgen05.mma.cta_group::1.kind::f16 [%0], [a], b, %3, p;\n\t"
       "add.u32 a, %1, 24;\n\tadd.u64 b, %2, 384;\n\t"
       "tcgen05.mma.cta_group::1.kind::f16 [%0], [a], b, %3, p;\n\t"
-      "add.u32 a, %1, 32;\n\tadd.u64 b, %2, 512;\n\t"
+      "add.u32 a, %1, 64;\n\tadd.u64 b, %2, 512;\n\t"
       "tcgen05.mma.cta_group::1.kind::f16 [%0], [a], b, %3, p;\n\t"
-      "add.u32 a, %1, 40;\n\tadd.u64 b, %2, 640;\n\t"
+      "add.u32 a, %1, 72;\n\tadd.u64 b, %2, 640;\n\t"
       "tcgen05.mma.cta_group::1.kind::f16 [%0], [a], b, %3, p;\n\t"
-      "add.u32 a, %1, 48;\n\tadd.u64 b, %2, 768;\n\t"
+      "add.u32 a, %1, 80;\n\tadd.u64 b, %2, 768;\n\t"
       "tcgen05.mma.cta_group::1.kind::f16 [%0], [a], b, %3, p;\n\t"
-      "add.u32 a, %1, 56;\n\tadd.u64 b, %2, 896;\n\t"
+      "add.u32 a, %1, 88;\n\tadd.u64 b, %2, 896;\n\t"
       "tcgen05.mma.cta_group::1.kind::f16 [%0], [a], b, %3, p;\n\t}"
       ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
       : "memory");
