@@ -1,5 +1,5 @@
 // Byte-exact cache movement: append of one block into the monolithic ring and/or the per-archetype
-// buffers, the split of the monolithic cache (one launch per cached block), and the export of one
+// buffers, the split of the monolithic cache (one launch, one grid row per cached block), and the export of one
 // head's logical content.  All copies move 16-byte chunks; a thread handles a few chunks of K and of V
 // so that enough loads are in flight to cover HBM latency.
 #pragma once
@@ -30,72 +30,86 @@ struct RouteParams {
   const int32_t* sp_nc;    // [T_f]: tokens per frame in the token's cell
   int32_t L, H, chunks;    // chunks = d / 8
   int32_t tokens_per_frame, frames_per_block, n_blocks;
-  int32_t slot;            // destination ring slot
   int32_t n_sink;
-  int32_t copy_mono, copy_sink, copy_dummy, copy_window;
+  int32_t copy_mono, copy_window;
+  // blockIdx.y selects the source block: it is read at src + src_stride * slots[y] (stride 0: the caller's block)
+  // and lands in ring slot slots[y]; only source sink_src feeds the Sink heads, only dummy_src the Dummy heads
+  long long src_stride;    // in 16-byte chunks
+  int32_t sink_src, dummy_src;
+  int8_t slots[MAX_BLOCKS];
   int8_t cls[MAX_HEADS];   // archetype per original head (CLS_NONE before the split)
   int8_t idx[MAX_HEADS];   // index of the head inside its archetype group
 };
 
-__device__ __forceinline__ long long route_dst(const RouteParams& p, int t, int h, int c, uint4** k, uint4** v) {
-  const int cls = p.cls[h], idx = p.idx[h];
-  if (cls == CLS_SINK) {
-    if (!p.copy_sink) return -1;
-    *k = p.sd_k; *v = p.sd_v;
-    return (static_cast<long long>(idx) * p.L + t) * p.chunks + c;
-  }
-  if (cls == CLS_DUMMY) {
-    if (!p.copy_dummy) return -1;
-    *k = p.sd_k; *v = p.sd_v;
-    return (static_cast<long long>(p.n_sink + idx) * p.L + t) * p.chunks + c;
-  }
-  if (!p.copy_window) return -1;
-  if (cls == CLS_GLOBAL) {
-    *k = p.g_k; *v = p.g_v;
-    return ((static_cast<long long>(idx) * p.n_blocks + p.slot) * p.L + t) * p.chunks + c;
-  }
-  if (cls == CLS_SPATIAL) {
-    *k = p.sp_k; *v = p.sp_v;
-    const int f = t / p.tokens_per_frame, pos = t - f * p.tokens_per_frame;
-    const long long row = static_cast<long long>(idx) * p.n_blocks * p.L + p.sp_base[pos] +
-                          static_cast<long long>(p.slot * p.frames_per_block + f) * p.sp_nc[pos];
-    return row * p.chunks + c;
-  }
-  return -1;
-}
-
 constexpr int ROUTE_UNROLL = 4;
 
-__global__ void __launch_bounds__(256) route_block_kernel(const RouteParams p) {
-  const long long per_token = static_cast<long long>(p.H) * p.chunks;
-  const long long total = per_token * p.L;
-  const long long stride = static_cast<long long>(gridDim.x) * blockDim.x;
-  for (long long g0 = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; g0 < total;
-       g0 += stride * ROUTE_UNROLL) {
+// Threads of a block are laid over (token, head, 16-byte chunk) of consecutive source tokens, so a thread's head -
+// and with it where its chunks go, or that nobody keeps them - is fixed for the whole launch; only the token
+// advances.  blockDim.x must be a multiple of H * chunks.
+__global__ void __launch_bounds__(1024) route_block_kernel(const RouteParams p) {
+  const int per_token = p.H * p.chunks;
+  const int tokens_per_iter = blockDim.x / per_token;
+  const int tl = threadIdx.x / per_token, hc = threadIdx.x - tl * per_token;
+  const int h = hc / p.chunks, c = hc - h * p.chunks;
+  const int src = blockIdx.y, slot = p.slots[src];
+  const long long total = static_cast<long long>(per_token) * p.L;
+  const uint4* src_k = p.src_k + p.src_stride * slot;
+  const uint4* src_v = p.src_v + p.src_stride * slot;
+  const int cls = p.cls[h], idx = p.idx[h];
+  // destination of this thread's chunks: base + t * chunks for the row-major buffers
+  uint4 *dk = nullptr, *dv = nullptr;
+  long long base = 0;
+  bool spatial = false;
+  if (cls == CLS_SINK && src == p.sink_src) {
+    dk = p.sd_k; dv = p.sd_v;
+    base = static_cast<long long>(idx) * p.L * p.chunks + c;
+  } else if (cls == CLS_DUMMY && src == p.dummy_src) {
+    dk = p.sd_k; dv = p.sd_v;
+    base = static_cast<long long>(p.n_sink + idx) * p.L * p.chunks + c;
+  } else if (cls == CLS_GLOBAL && p.copy_window) {
+    dk = p.g_k; dv = p.g_v;
+    base = (static_cast<long long>(idx) * p.n_blocks + slot) * p.L * p.chunks + c;
+  } else if (cls == CLS_SPATIAL && p.copy_window) {
+    dk = p.sp_k; dv = p.sp_v;
+    base = static_cast<long long>(idx) * p.n_blocks * p.L;  // in rows; the rest depends on the token
+    spatial = true;
+  }
+  if (!dk && !p.copy_mono) return;  // chunks nobody keeps (Sink / Dummy heads of the other blocks) are never loaded
+  const int t_stride = gridDim.x * tokens_per_iter;
+  for (int t0 = blockIdx.x * tokens_per_iter + tl; t0 < p.L; t0 += t_stride * ROUTE_UNROLL) {
     uint4 kv[ROUTE_UNROLL], vv[ROUTE_UNROLL];
+    int sb[ROUTE_UNROLL], sn[ROUTE_UNROLL];
 #pragma unroll
     for (int u = 0; u < ROUTE_UNROLL; ++u) {
-      const long long g = g0 + u * stride;
-      if (g < total) {
-        kv[u] = __ldcs(p.src_k + g);
-        vv[u] = __ldcs(p.src_v + g);
+      const int t = t0 + u * t_stride;
+      if (t < p.L) {
+        const long long g = static_cast<long long>(t) * per_token + hc;
+        kv[u] = __ldcs(src_k + g);
+        vv[u] = __ldcs(src_v + g);
+        if (spatial) {
+          const int pos = t % p.tokens_per_frame;
+          sb[u] = p.sp_base[pos];
+          sn[u] = p.sp_nc[pos];
+        }
       }
     }
 #pragma unroll
     for (int u = 0; u < ROUTE_UNROLL; ++u) {
-      const long long g = g0 + u * stride;
-      if (g >= total) continue;
-      const int t = static_cast<int>(g / per_token);
-      const int rem = static_cast<int>(g - t * per_token);
-      const int h = rem / p.chunks, c = rem - h * p.chunks;
+      const int t = t0 + u * t_stride;
+      if (t >= p.L) continue;
       if (p.copy_mono) {
-        const long long m = static_cast<long long>(p.slot) * total + g;
+        const long long m = static_cast<long long>(slot) * total + static_cast<long long>(t) * per_token + hc;
         p.mono_k[m] = kv[u];
         p.mono_v[m] = vv[u];
       }
-      uint4 *dk = nullptr, *dv = nullptr;
-      const long long d = route_dst(p, t, h, c, &dk, &dv);
-      if (d >= 0) {
+      if (dk) {
+        long long d;
+        if (spatial) {
+          const int f = t / p.tokens_per_frame;
+          d = (base + sb[u] + static_cast<long long>(slot * p.frames_per_block + f) * sn[u]) * p.chunks + c;
+        } else {
+          d = base + static_cast<long long>(t) * p.chunks;
+        }
         dk[d] = kv[u];
         dv[d] = vv[u];
       }

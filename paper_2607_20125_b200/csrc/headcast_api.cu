@@ -499,11 +499,14 @@ void fill_route(headcast_ctx* c, RouteParams& r) {
   }
 }
 
-int launch_route(headcast_ctx* c, const RouteParams& r, cudaStream_t st) {
-  const long long total = static_cast<long long>(r.L) * r.H * r.chunks;
-  const long long per_block = 256LL * ROUTE_UNROLL;
-  const int blocks = static_cast<int>(std::min<long long>((total + per_block - 1) / per_block, c->n_sm * 8LL));
-  route_block_kernel<<<std::max(1, blocks), 256, 0, st>>>(r);
+int launch_route(headcast_ctx* c, const RouteParams& r, int n_src, cudaStream_t st) {
+  const int per_token = r.H * r.chunks;  // <= 64 heads * 16 chunks = 1024
+  const int tokens_per_iter = std::max(1, 256 / per_token);
+  const int threads = tokens_per_iter * per_token;
+  const int resident = std::max(1, 2048 / threads);  // blocks per SM
+  const int per_src = std::max(1, (c->n_sm * resident + n_src - 1) / n_src);
+  const int needed = (r.L + tokens_per_iter * ROUTE_UNROLL - 1) / (tokens_per_iter * ROUTE_UNROLL);
+  route_block_kernel<<<dim3(std::max(1, std::min(needed, per_src)), n_src), threads, 0, st>>>(r);
   HC_CUDA(c, cudaGetLastError());
   ++c->launches;
   return HC_OK;
@@ -693,12 +696,13 @@ int headcast_append(headcast_ctx* c, const void* k_new, const void* v_new, void*
   fill_route(c, r);
   r.src_k = static_cast<const uint4*>(k_new);
   r.src_v = static_cast<const uint4*>(v_new);
-  r.slot = slot;
+  r.slots[0] = static_cast<int8_t>(slot);
+  r.src_stride = 0;
   r.copy_mono = c->mono_k != nullptr;
-  r.copy_sink = 0;  // frozen
-  r.copy_dummy = c->state == STATE_SPLIT;
+  r.sink_src = -1;  // frozen
+  r.dummy_src = (c->state == STATE_SPLIT) ? 0 : -1;
   r.copy_window = c->state == STATE_SPLIT;
-  int rc = launch_route(c, r, st);
+  int rc = launch_route(c, r, 1, st);
   if (rc != HC_OK) return rc;
   c->slots.swap(next);
   return HC_OK;
@@ -851,19 +855,19 @@ int headcast_split_cache(headcast_ctx* c, void* stream) {
   c->g_v = g_elems ? c->arena_v + sd_elems : nullptr;
   c->sp_k = sp_elems ? c->arena_k + sd_elems + g_elems : nullptr;
   c->sp_v = sp_elems ? c->arena_v + sd_elems + g_elems : nullptr;
-  const size_t block_elems = static_cast<size_t>(c->L) * c->H * c->D;
-  for (size_t i = 0; i < c->slots.size(); ++i) {
+  {
+    // one launch: grid row i gathers cached block i (ring slot slots[i]) out of the monolithic cache
     RouteParams r;
     fill_route(c, r);
-    const int slot = c->slots[i];
-    r.src_k = reinterpret_cast<const uint4*>(c->mono_k + slot * block_elems);
-    r.src_v = reinterpret_cast<const uint4*>(c->mono_v + slot * block_elems);
-    r.slot = slot;
+    r.src_k = reinterpret_cast<const uint4*>(c->mono_k);
+    r.src_v = reinterpret_cast<const uint4*>(c->mono_v);
+    r.src_stride = static_cast<long long>(c->L) * c->H * c->CH;
+    for (size_t i = 0; i < c->slots.size(); ++i) r.slots[i] = static_cast<int8_t>(c->slots[i]);
     r.copy_mono = 0;
-    r.copy_sink = (i == 0);
-    r.copy_dummy = (i + 1 == c->slots.size());
+    r.sink_src = 0;
+    r.dummy_src = static_cast<int32_t>(c->slots.size()) - 1;
     r.copy_window = 1;
-    int rc = launch_route(c, r, st);
+    int rc = launch_route(c, r, static_cast<int>(c->slots.size()), st);
     if (rc != HC_OK) return rc;
   }
   if (!c->cfg.keep_monolithic) {
