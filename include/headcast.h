@@ -163,6 +163,17 @@ int headcast_last_attention_kernel_ms(headcast_ctx* ctx, float* ms_host);
 int headcast_set_tracing(headcast_ctx* ctx, int32_t enable);
 int headcast_read_trace(headcast_ctx* ctx, int64_t* rows_host, int32_t capacity, int32_t* n_items_host);
 
+/* Host-only (no GPU needed): the work list headcast_attend (dense = 0, labels_host[H] given) or headcast_full_attend
+ * (dense = 1) would run with n_filled cached blocks on n_ctas persistent CTAs.  Every item is 16 int32:
+ * head, Spatial cell or -1, first query (token, or packed index inside the cell) of query tile 0 and 1, valid rows of
+ * tile 0 and 1, buffer (0 monolithic, 1 Sink-Dummy, 2 Global, 3 Spatial), element column, first key row, row stride
+ * between key segments, keys per segment, 128-key tiles per segment, first and one-past-last tile of this item,
+ * output mode (0 final, 1 partial to be merged), partial slot.  items_host has room for `capacity` items,
+ * cta_first_host for n_ctas + 1 entries (items of CTA b are [cta_first[b], cta_first[b+1])); either may be NULL. */
+int headcast_plan_schedule(const headcast_config* cfg, const int32_t* labels_host, int32_t n_filled, int32_t n_ctas,
+                           int32_t dense, int32_t* items_host, int32_t capacity, int32_t* n_items_host,
+                           int32_t* cta_first_host);
+
 /* Synchronises `stream` and reports a device-side status raised by any earlier kernel of this context
  * (HC_ERR_TIMEOUT if a bounded wait expired). */
 int headcast_check(headcast_ctx* ctx, void* stream);

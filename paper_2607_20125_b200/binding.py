@@ -23,7 +23,7 @@ EXPORTS = ("headcast_default_config", "headcast_create", "headcast_destroy", "he
            "headcast_launch_count", "headcast_attend_flops", "headcast_check", "headcast_last_error",
            "headcast_set_kernel_timing", "headcast_last_attention_kernel_ms", "headcast_set_tracing",
            "headcast_read_trace", "headcast_dense_attend_noalloc", "headcast_noalloc_status",
-           "headcast_noalloc_last_error")
+           "headcast_noalloc_last_error", "headcast_plan_schedule")
 
 
 class Config(C.Structure):
@@ -76,6 +76,7 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.headcast_read_trace.argtypes = [vp, C.POINTER(C.c_int64), C.c_int32, i32p]
     lib.headcast_dense_attend_noalloc.argtypes = [vp, vp, vp, vp, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_float, vp]
     lib.headcast_noalloc_status.argtypes = [vp]
+    lib.headcast_plan_schedule.argtypes = [C.POINTER(Config), i32p, C.c_int32, C.c_int32, C.c_int32, i32p, C.c_int32, i32p, i32p]
     lib.headcast_noalloc_last_error.argtypes = []
     lib.headcast_noalloc_last_error.restype = C.c_char_p
     lib.headcast_last_error.argtypes = [vp]
@@ -101,6 +102,29 @@ def _stream() -> int:
 def _ptr(t) -> int:
     assert t.is_cuda and t.is_contiguous(), "tensors handed to the library must be contiguous CUDA tensors"
     return t.data_ptr()
+
+
+ITEM_FIELDS = ("head", "cell", "q_start0", "q_start1", "q_count0", "q_count1", "kv_map", "kv_x0", "kv_row0", "seg_stride",
+               "seg_len", "tiles_per_seg", "tile_begin", "tile_end", "out_mode", "out_slot")
+
+
+def plan_schedule(cfg: Config, labels: Optional[Sequence[int]], n_filled: int, n_ctas: int = 148, dense: bool = False):
+    """Host-only: the work list of headcast_attend / headcast_full_attend as (items [n, 16] int32 with columns
+    ITEM_FIELDS, cta_first [n_ctas + 1] int32)."""
+    import numpy as np
+    lib = load_library()
+    lab = None if labels is None else (C.c_int32 * cfg.n_heads)(*[int(v) for v in labels])
+    n = C.c_int32()
+    rc = lib.headcast_plan_schedule(C.byref(cfg), lab, n_filled, n_ctas, int(dense), None, 0, C.byref(n), None)
+    if rc != 0:
+        raise HeadCastError(rc, "headcast_plan_schedule")
+    items = np.zeros((max(n.value, 1), 16), dtype=np.int32)
+    first = np.zeros(n_ctas + 1, dtype=np.int32)
+    rc = lib.headcast_plan_schedule(C.byref(cfg), lab, n_filled, n_ctas, int(dense), items.ctypes.data_as(C.POINTER(C.c_int32)),
+                                    n.value, C.byref(n), first.ctypes.data_as(C.POINTER(C.c_int32)))
+    if rc != 0:
+        raise HeadCastError(rc, "headcast_plan_schedule")
+    return items[: n.value], first
 
 
 def dense_attend_noalloc(q, k, v, out, softmax_scale: float = 0.0) -> None:

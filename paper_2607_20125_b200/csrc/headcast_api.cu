@@ -216,18 +216,20 @@ WorkItem range_item(int head, int map, int x0, long long row0, int n_keys) {
 }
 
 // Cost model of the scheduler, in units of the time one key tile takes with both query tiles in flight
-// (fitted to per-item timings from headcast_read_trace on B200): a lone query tile still needs 0.86 of that
+// (fitted to per-item timings from headcast_read_trace on B200): a lone query tile still needs 0.82 of that
 // because the chain S -> softmax -> P -> next S is latency bound; every item pays for its query load, pipeline
 // fill and epilogue; a partial result costs an extra round trip through global memory.
-constexpr double TILE_COST_PAIR = 1.0, TILE_COST_SINGLE = 0.86;
-constexpr double ITEM_OVERHEAD = 3.5;
+constexpr double TILE_COST_PAIR = 1.0, TILE_COST_SINGLE = 0.82;
+constexpr double ITEM_OVERHEAD = 3.5, ITEM_OVERHEAD_SINGLE = 2.5;
 constexpr double PARTIAL_EXTRA = 1.0;
 constexpr int MIN_PART_TILES = 4;  // never cut a key range into pieces shorter than this
 
 double tile_cost(const WorkItem& w) { return w.q_count[1] > 0 ? TILE_COST_PAIR : TILE_COST_SINGLE; }
 
+double item_overhead(const WorkItem& w) { return w.q_count[1] > 0 ? ITEM_OVERHEAD : ITEM_OVERHEAD_SINGLE; }
+
 double item_cost(const WorkItem& w) {
-  return tile_cost(w) * (w.tile_end - w.tile_begin) + ITEM_OVERHEAD + (w.out_mode == OUT_PARTIAL ? PARTIAL_EXTRA : 0.0);
+  return tile_cost(w) * (w.tile_end - w.tile_begin) + item_overhead(w) + (w.out_mode == OUT_PARTIAL ? PARTIAL_EXTRA : 0.0);
 }
 
 // Assigns work to the persistent CTAs (one per SM).
@@ -244,70 +246,85 @@ void finalize_schedule(headcast_ctx* c, Schedule& s, std::vector<Proto>& protos,
   std::stable_sort(protos.begin(), protos.end(),
                    [](const Proto& a, const Proto& b) { return item_cost(a.w) > item_cost(b.w); });
   if (allow_split) {
-    double total = 0.0;
-    for (const Proto& p : protos) total += item_cost(p.w);
-    const double slack = 0.02 * total / n_cta;
-    int cta = 0;
-    double unassigned = total;  // tile-times not yet placed; the share of each further CTA is re-derived from it
-    double room = total / n_cta;
-    auto next_cta = [&]() {
-      if (cta + 1 < n_cta) {
-        ++cta;
-        room = unassigned / (n_cta - cta);
-      } else {
-        room = 1e30;
-      }
-    };
+    // Lay the items end to end and give every CTA the same share Q of the line, cutting the item that straddles a
+    // boundary.  Cuts add cost of their own (a second query load and epilogue, partial results), so the share that
+    // makes everything fit on n_cta CTAs is found by bisection: lay_out(Q) reports the load of the last CTA.
+    double base_total = 0.0, largest = 0.0;
     for (const Proto& p : protos) {
-      const int n_q = p.w.q_count[1] > 0 ? 2 : 1;
-      const double per_tile = tile_cost(p.w);
-      std::vector<std::pair<int, WorkItem>> parts;  // (cta, piece)
-      int begin = 0;
-      while (begin < p.n_tiles) {
-        const int left = p.n_tiles - begin;
-        const double need = per_tile * left + ITEM_OVERHEAD;
-        int take = left;
-        if (need > room + slack) {
-          const int can = static_cast<int>(std::floor((room - ITEM_OVERHEAD - PARTIAL_EXTRA) / per_tile));
-          if (can < MIN_PART_TILES) {
-            next_cta();
-            continue;
-          }
-          if (left - can >= MIN_PART_TILES) take = can;
-        }
-        WorkItem w = p.w;
-        w.tile_begin = begin;
-        w.tile_end = begin + take;
-        parts.push_back(std::make_pair(cta, w));
-        const bool cut = (take < left) || begin > 0;
-        room -= per_tile * take + ITEM_OVERHEAD + (cut ? PARTIAL_EXTRA : 0.0);
-        unassigned -= per_tile * take + (begin == 0 ? ITEM_OVERHEAD : 0.0);
-        begin += take;
-        if (room < ITEM_OVERHEAD + MIN_PART_TILES) next_cta();
-      }
-      if (parts.size() == 1) {
-        bins[parts[0].first].push_back(parts[0].second);
-        continue;
-      }
-      const int first_slot = s.n_slots;
-      for (auto& pr : parts) {
-        pr.second.out_mode = OUT_PARTIAL;
-        pr.second.out_slot = s.n_slots++;
-        bins[pr.first].push_back(pr.second);
-      }
-      for (int t = 0; t < n_q; ++t) {
-        CombineEntry e;
-        e.head = p.w.head;
-        e.cell = p.w.cell;
-        e.q_start = p.w.q_start[t];
-        e.q_count = p.w.q_count[t];
-        e.first_slot = first_slot;
-        e.n_parts = static_cast<int32_t>(parts.size());
-        e.sub = t;
-        e.pad = 0;
-        s.combine.push_back(e);
-      }
+      base_total += item_cost(p.w);
+      largest = std::max(largest, item_cost(p.w));
     }
+    auto lay_out = [&](double quota) -> double {
+      for (auto& bin : bins) bin.clear();
+      s.combine.clear();
+      s.n_slots = 0;
+      int cta = 0;
+      double room = quota, last_load = 0.0;
+      auto next_cta = [&]() {
+        if (cta + 1 < n_cta) {
+          ++cta;
+          room = quota;
+        }
+      };
+      for (const Proto& p : protos) {
+        const int n_q = p.w.q_count[1] > 0 ? 2 : 1;
+        const double per_tile = tile_cost(p.w), overhead = item_overhead(p.w);
+        std::vector<std::pair<int, WorkItem>> parts;  // (cta, piece)
+        int begin = 0;
+        while (begin < p.n_tiles) {
+          const int left = p.n_tiles - begin;
+          const double need = per_tile * left + overhead + (begin > 0 ? PARTIAL_EXTRA : 0.0);
+          int take = left;
+          if (need > room && cta + 1 < n_cta) {
+            const int can = static_cast<int>(std::floor((room - overhead - PARTIAL_EXTRA) / per_tile));
+            if (can < MIN_PART_TILES || left - can < MIN_PART_TILES) {  // no piece worth cutting fits here
+              next_cta();
+              continue;
+            }
+            take = can;
+          }
+          WorkItem w = p.w;
+          w.tile_begin = begin;
+          w.tile_end = begin + take;
+          parts.push_back(std::make_pair(cta, w));
+          const bool cut = (take < left) || begin > 0;
+          const double cost = per_tile * take + overhead + (cut ? PARTIAL_EXTRA : 0.0);
+          room -= cost;
+          if (cta == n_cta - 1) last_load += cost;
+          begin += take;
+        }
+        if (parts.size() == 1) {
+          bins[parts[0].first].push_back(parts[0].second);
+          continue;
+        }
+        const int first_slot = s.n_slots;
+        for (auto& pr : parts) {
+          pr.second.out_mode = OUT_PARTIAL;
+          pr.second.out_slot = s.n_slots++;
+          bins[pr.first].push_back(pr.second);
+        }
+        for (int t = 0; t < n_q; ++t) {
+          CombineEntry e;
+          e.head = p.w.head;
+          e.cell = p.w.cell;
+          e.q_start = p.w.q_start[t];
+          e.q_count = p.w.q_count[t];
+          e.first_slot = first_slot;
+          e.n_parts = static_cast<int32_t>(parts.size());
+          e.sub = t;
+          e.pad = 0;
+          s.combine.push_back(e);
+        }
+      }
+      return last_load;
+    };
+    double lo = base_total / n_cta, hi = base_total / n_cta + largest + ITEM_OVERHEAD + PARTIAL_EXTRA;
+    while (lay_out(hi) > hi) hi *= 1.25;
+    for (int iter = 0; iter < 24 && hi - lo > 0.25; ++iter) {
+      const double mid = 0.5 * (lo + hi);
+      if (lay_out(mid) <= mid) hi = mid; else lo = mid;
+    }
+    lay_out(hi);
   } else {
     typedef std::pair<double, int> Load;
     std::priority_queue<Load, std::vector<Load>, std::greater<Load>> pq;
@@ -533,6 +550,61 @@ void assign_classes(headcast_ctx* c) {
 
 }  // namespace
 
+// Host-only half of headcast_create: validates cfg and fills sizes, cell geometry and the cell-major token tables.
+static int init_host(headcast_ctx* c, const headcast_config* cfg, std::vector<int32_t>& sp_base, std::vector<int32_t>& sp_nc) {
+  if (cfg->n_heads < 1 || cfg->n_heads > MAX_HEADS || (cfg->head_dim != 64 && cfg->head_dim != 128) ||
+      cfg->grid_h < 1 || cfg->grid_w < 1 || cfg->frames_per_block < 1 || cfg->n_blocks < 2 ||
+      cfg->n_blocks > MAX_BLOCKS || cfg->cell_h < 1 || cfg->cell_w < 1 || cfg->proxy_radius < 0 ||
+      !(cfg->softmax_scale >= 0.0f))
+    return HC_ERR_INVALID_ARG;
+  const long long L = static_cast<long long>(cfg->frames_per_block) * cfg->grid_h * cfg->grid_w;
+  if (L * cfg->n_blocks * cfg->n_heads * cfg->head_dim >= (1LL << 40) || L * cfg->n_blocks * cfg->n_heads >= (1LL << 31))
+    return HC_ERR_INVALID_ARG;
+  c->cfg = *cfg;
+  c->H = cfg->n_heads;
+  c->D = cfg->head_dim;
+  c->G_h = cfg->grid_h;
+  c->G_w = cfg->grid_w;
+  c->F_b = cfg->frames_per_block;
+  c->T_f = cfg->grid_h * cfg->grid_w;
+  c->L = static_cast<int>(L);
+  c->n_blk = cfg->n_blocks;
+  c->CH = c->D / 8;
+  c->scale = cfg->softmax_scale > 0.f ? cfg->softmax_scale : 1.0f / std::sqrt(static_cast<float>(c->D));
+  c->row_edges = (cfg->row_edges_host && cfg->n_row_edges > 0)
+                     ? std::vector<int>(cfg->row_edges_host, cfg->row_edges_host + cfg->n_row_edges)
+                     : default_edges(c->G_h, cfg->cell_h);
+  c->col_edges = (cfg->col_edges_host && cfg->n_col_edges > 0)
+                     ? std::vector<int>(cfg->col_edges_host, cfg->col_edges_host + cfg->n_col_edges)
+                     : default_edges(c->G_w, cfg->cell_w);
+  c->cfg.row_edges_host = c->cfg.col_edges_host = nullptr;
+  if (!edges_ok(c->row_edges, c->G_h) || !edges_ok(c->col_edges, c->G_w)) return HC_ERR_INVALID_ARG;
+  c->labels.assign(c->H, HC_GLOBAL);
+  for (int h = 0; h < c->H; ++h) {
+    c->cls[h] = CLS_NONE;
+    c->idx[h] = 0;
+  }
+  // deployed cells and the cell-major token order of the Spatial buffers
+  sp_base.assign(c->T_f, 0);
+  sp_nc.assign(c->T_f, 0);
+  int tok_off = 0;
+  for (size_t i = 0; i + 1 < c->row_edges.size(); ++i)
+    for (size_t j = 0; j + 1 < c->col_edges.size(); ++j) {
+      CellGeom g = {c->row_edges[i], c->col_edges[j], c->row_edges[i + 1] - c->row_edges[i],
+                    c->col_edges[j + 1] - c->col_edges[j]};
+      c->cells.push_back(g);
+      c->cell_tok_off.push_back(tok_off);
+      for (int dy = 0; dy < g.ch; ++dy)
+        for (int dx = 0; dx < g.cw; ++dx) {
+          const int pos = (g.y0 + dy) * c->G_w + g.x0 + dx;
+          sp_base[pos] = c->n_blk * c->F_b * tok_off + dy * g.cw + dx;
+          sp_nc[pos] = g.ch * g.cw;
+        }
+      tok_off += g.ch * g.cw;
+    }
+  return HC_OK;
+}
+
 // =====================================================================================================
 extern "C" {
 
@@ -552,60 +624,16 @@ void headcast_default_config(headcast_config* cfg) {
 int headcast_create(const headcast_config* cfg, headcast_ctx** out) {
   if (!cfg || !out) return HC_ERR_INVALID_ARG;
   *out = nullptr;
-  if (cfg->n_heads < 1 || cfg->n_heads > MAX_HEADS || (cfg->head_dim != 64 && cfg->head_dim != 128) ||
-      cfg->grid_h < 1 || cfg->grid_w < 1 || cfg->frames_per_block < 1 || cfg->n_blocks < 2 ||
-      cfg->n_blocks > MAX_BLOCKS || cfg->cell_h < 1 || cfg->cell_w < 1 || cfg->proxy_radius < 0 ||
-      !(cfg->softmax_scale >= 0.0f))
-    return HC_ERR_INVALID_ARG;
-  const long long L = static_cast<long long>(cfg->frames_per_block) * cfg->grid_h * cfg->grid_w;
-  if (L * cfg->n_blocks * cfg->n_heads * cfg->head_dim >= (1LL << 40) || L * cfg->n_blocks * cfg->n_heads >= (1LL << 31))
-    return HC_ERR_INVALID_ARG;
   headcast_ctx* c = new (std::nothrow) headcast_ctx();
   if (!c) return HC_ERR_NOMEM;
-  c->cfg = *cfg;
-  c->H = cfg->n_heads;
-  c->D = cfg->head_dim;
-  c->G_h = cfg->grid_h;
-  c->G_w = cfg->grid_w;
-  c->F_b = cfg->frames_per_block;
-  c->T_f = cfg->grid_h * cfg->grid_w;
-  c->L = static_cast<int>(L);
-  c->n_blk = cfg->n_blocks;
-  c->CH = c->D / 8;
-  c->scale = cfg->softmax_scale > 0.f ? cfg->softmax_scale : 1.0f / std::sqrt(static_cast<float>(c->D));
-  c->row_edges = (cfg->row_edges_host && cfg->n_row_edges > 0)
-                     ? std::vector<int>(cfg->row_edges_host, cfg->row_edges_host + cfg->n_row_edges)
-                     : default_edges(c->G_h, cfg->cell_h);
-  c->col_edges = (cfg->col_edges_host && cfg->n_col_edges > 0)
-                     ? std::vector<int>(cfg->col_edges_host, cfg->col_edges_host + cfg->n_col_edges)
-                     : default_edges(c->G_w, cfg->cell_w);
-  c->cfg.row_edges_host = c->cfg.col_edges_host = nullptr;
-  if (!edges_ok(c->row_edges, c->G_h) || !edges_ok(c->col_edges, c->G_w)) {
-    delete c;
-    return HC_ERR_INVALID_ARG;
-  }
-  c->labels.assign(c->H, HC_GLOBAL);
-  for (int h = 0; h < c->H; ++h) {
-    c->cls[h] = CLS_NONE;
-    c->idx[h] = 0;
-  }
-  // deployed cells and the cell-major token order of the Spatial buffers
-  std::vector<int32_t> sp_base(c->T_f), sp_nc(c->T_f);
-  int tok_off = 0;
-  for (size_t i = 0; i + 1 < c->row_edges.size(); ++i)
-    for (size_t j = 0; j + 1 < c->col_edges.size(); ++j) {
-      CellGeom g = {c->row_edges[i], c->col_edges[j], c->row_edges[i + 1] - c->row_edges[i],
-                    c->col_edges[j + 1] - c->col_edges[j]};
-      c->cells.push_back(g);
-      c->cell_tok_off.push_back(tok_off);
-      for (int dy = 0; dy < g.ch; ++dy)
-        for (int dx = 0; dx < g.cw; ++dx) {
-          const int pos = (g.y0 + dy) * c->G_w + g.x0 + dx;
-          sp_base[pos] = c->n_blk * c->F_b * tok_off + dy * g.cw + dx;
-          sp_nc[pos] = g.ch * g.cw;
-        }
-      tok_off += g.ch * g.cw;
+  std::vector<int32_t> sp_base, sp_nc;
+  {
+    const int rc = init_host(c, cfg, sp_base, sp_nc);
+    if (rc != HC_OK) {
+      delete c;
+      return rc;
     }
+  }
   int dev = 0;
   cudaDeviceProp prop;
   if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess) {
@@ -1011,6 +1039,36 @@ int headcast_read_timeline(headcast_ctx* c, int64_t* out_host /* [64][16] */) {
   return HC_OK;
 }
 #endif
+
+int headcast_plan_schedule(const headcast_config* cfg, const int32_t* labels_host, int32_t n_filled, int32_t n_ctas,
+                           int32_t dense, int32_t* items_host, int32_t capacity, int32_t* n_items_host,
+                           int32_t* cta_first_host) {
+  if (!cfg || !n_items_host || n_filled < 1 || n_ctas < 1 || n_ctas > 4096) return HC_ERR_INVALID_ARG;
+  headcast_ctx c;
+  std::vector<int32_t> sp_base, sp_nc;
+  int rc = init_host(&c, cfg, sp_base, sp_nc);
+  if (rc != HC_OK) return rc;
+  if (n_filled > c.n_blk) return HC_ERR_INVALID_ARG;
+  c.n_sm = n_ctas;
+  for (int i = 0; i < n_filled; ++i) c.slots.push_back(i);
+  Schedule s;
+  if (dense) {
+    build_dense_schedule(&c, s, OUT_BF16, true);
+  } else {
+    if (!labels_host) return HC_ERR_INVALID_ARG;
+    for (int h = 0; h < c.H; ++h)
+      if (labels_host[h] < 0 || labels_host[h] > 3) return HC_ERR_INVALID_ARG;
+    c.labels.assign(labels_host, labels_host + c.H);
+    assign_classes(&c);
+    build_headcast_schedule(&c, s);
+  }
+  *n_items_host = static_cast<int32_t>(s.items.size());
+  static_assert(sizeof(WorkItem) == 16 * sizeof(int32_t), "work items are exported as 16 int32 each");
+  if (items_host)
+    std::memcpy(items_host, s.items.data(), std::min<size_t>(s.items.size(), capacity) * sizeof(WorkItem));
+  if (cta_first_host) std::copy(s.cta_first.begin(), s.cta_first.end(), cta_first_host);
+  return HC_OK;
+}
 
 int headcast_check(headcast_ctx* c, void* stream) {
   if (!c) return HC_ERR_INVALID_ARG;
