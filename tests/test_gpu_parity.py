@@ -234,3 +234,69 @@ def test_480p_sampled_rows():
     rows = synth.sample_rows(w, n_random=128)
     p = run_pipeline(w, fill=7, extra=1, rows=rows)
     assert abs(p.hc.attend_flops(False) / 1e9 - 312.5) < 0.5 and abs(p.hc.attend_flops(True) / 1e9 - 942.0) < 0.5
+
+
+def test_classify_480p_labels_and_sampled_scores():
+    # full-size classification on the GPU; the oracle scores a sample of rows (its statistics are those of the sample,
+    # so only quantities that do not depend on the row set are compared tightly)
+    w = synth.wan("480p")
+    p = Pair(w)
+    p.append(7)
+    q = synth.make_q(w, 6, 0)
+    labels, scores = p.hc.classify(to_dev(q))
+    rows = synth.sample_rows(w, n_random=64)[::3]
+    want_labels, want = orc.classify(q, p.cache, p.geom, rows=rows)
+    assert tuple(labels) == tuple(want_labels) == tuple(w.labels)
+    d = np.abs(scores.astype(np.float64) - want)
+    assert d[:, [0, 1, 2]].max() <= 0.06 and d[:, [6, 7, 8, 9]].max() <= 0.06, d  # sample vs population means
+
+
+@pytest.mark.parametrize("res,n_random", [("720p", 48), ("1080p", 24)])
+def test_hd_grids_sampled_rows(res, n_random):
+    w = synth.wan(res)
+    rows = synth.sample_rows(w, n_random=n_random)[::5]
+    p = Pair(w, keep_monolithic=(res == "720p"))
+    p.append(7)
+    if res == "720p":
+        p.check_attention(dense=True, rows=rows)
+    p.hc.set_labels(w.labels)
+    p.hc.split_cache()
+    p.cache.split(w.labels)
+    for h in (0, 5, 11):  # one exported head per call keeps the host copies small
+        k, v = p.hc.export_cache(h)
+        ko, vo = p.cache.head_kv_bits(h)
+        assert np.array_equal(k, ko) and np.array_equal(v, vo)
+    p.check_attention(dense=False, rows=rows)
+    p.append()
+    p.check_attention(dense=False, rows=rows, step=1)
+
+
+def test_rollout_sequence_three_layers():
+    # the streaming schedule of a long rollout at small scale: per layer two warm-up blocks with dense attention, the third
+    # block appended and classified at its first denoise step, the split with 3 of 4 blocks cached, then generated
+    # blocks x 4 denoise steps with an append (and, once full, a roll) per block; cache checked bit-exactly every block
+    for layer in range(3):
+        w = synth.small(seed=synth.BASE_SEED + 101 * layer,
+                        labels=[(orc.GLOBAL, orc.SPATIAL, orc.SINK, orc.DUMMY, orc.SPATIAL, orc.GLOBAL),
+                                (orc.DUMMY, orc.GLOBAL, orc.SPATIAL, orc.SPATIAL, orc.SINK, orc.DUMMY),
+                                (orc.SPATIAL, orc.SINK, orc.GLOBAL, orc.DUMMY, orc.GLOBAL, orc.SPATIAL)][layer])
+        p = Pair(w)
+        rows = synth.sample_rows(w, n_random=40)
+        for _ in range(2):
+            p.append()
+            p.check_attention(dense=True, rows=rows)
+        p.append()
+        q = synth.make_q(w, 2, 0)
+        labels, _ = p.hc.classify(to_dev(q))
+        want_labels, _ = orc.classify(q, p.cache, p.geom, rows=rows)
+        assert tuple(labels) == tuple(want_labels) == tuple(w.labels)
+        p.hc.split_cache()
+        p.cache.split(labels)
+        p.check_cache()
+        for step in range(4):
+            p.check_attention(dense=False, rows=rows, step=step)
+        for block in range(4):
+            p.append()
+            p.check_cache()
+            for step in (0, 3):
+                p.check_attention(dense=False, rows=rows, step=step)
