@@ -130,11 +130,10 @@ def _oracle_state(w):
             cache.append(*synth.make_kv(w, b))
         cache.split(w.labels)
         q = synth.make_q(w, w.n_blocks - 1, 0)
-        rows = synth.sample_rows(w, n_random=4096)
-        rows = rows[np.random.default_rng(0).permutation(rows.size)]
+        rows = np.random.default_rng(0).permutation(w.block_tokens)  # seeded order over all query rows
         t0 = time.perf_counter()
-        orc.attend(q, cache, geom, rows=rows[:32])
-        per_row = (time.perf_counter() - t0) / 32
+        orc.attend(q, cache, geom, rows=rows[:256])
+        per_row = (time.perf_counter() - t0) / 256
         _ORACLE_STATE[w.name] = (orc, geom, cache, q, rows, per_row)
     return _ORACLE_STATE[w.name]
 
@@ -143,7 +142,7 @@ def cpu_baseline(w, target_s=12.0):
     """The oracle, as it stands, on a bounded sample of the same workload: head-specific attention for a few query
     rows of every head, extrapolated linearly to the whole block (rows are independent)."""
     orc, geom, cache, q, rows, per_row = _oracle_state(w)
-    n = int(max(32, min(rows.size, target_s / max(per_row, 1e-9))))
+    n = int(max(256, min(rows.size, target_s / max(per_row, 1e-9))))
     t0 = time.perf_counter()
     orc.attend(q, cache, geom, rows=rows[:n])
     dt = time.perf_counter() - t0
