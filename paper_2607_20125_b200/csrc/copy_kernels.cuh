@@ -37,21 +37,31 @@ struct RouteParams {
   long long src_stride;    // in 16-byte chunks
   int32_t sink_src, dummy_src;
   int8_t slots[MAX_BLOCKS];
+  // threads are laid over the heads somebody keeps: kept[k] lists them for source rows of kind k
+  // (0: feeds the Sink heads too, 1: the Dummy heads too, 2: both, 3: neither), n_kept[k] counts them
+  int8_t kind[MAX_BLOCKS];
+  int8_t n_kept[4];
+  int8_t kept[4][MAX_HEADS];
   int8_t cls[MAX_HEADS];   // archetype per original head (CLS_NONE before the split)
   int8_t idx[MAX_HEADS];   // index of the head inside its archetype group
 };
 
 constexpr int ROUTE_UNROLL = 4;
 
-// Threads of a block are laid over (token, head, 16-byte chunk) of consecutive source tokens, so a thread's head -
-// and with it where its chunks go, or that nobody keeps them - is fixed for the whole launch; only the token
-// advances.  blockDim.x must be a multiple of H * chunks.
+// Threads of a block are laid over (token, kept head, 16-byte chunk) of consecutive source tokens, so a thread's
+// head - and with it where its chunks go - is fixed for the whole launch and only the token advances; heads whose
+// chunks nobody keeps (Sink / Dummy heads of the other blocks) get no threads and are never loaded.
 __global__ void __launch_bounds__(1024) route_block_kernel(const RouteParams p) {
   const int per_token = p.H * p.chunks;
-  const int tokens_per_iter = blockDim.x / per_token;
-  const int tl = threadIdx.x / per_token, hc = threadIdx.x - tl * per_token;
-  const int h = hc / p.chunks, c = hc - h * p.chunks;
   const int src = blockIdx.y, slot = p.slots[src];
+  const int kind = p.kind[src];
+  const int kept_chunks = p.n_kept[kind] * p.chunks;
+  if (kept_chunks == 0) return;
+  const int tokens_per_iter = blockDim.x / kept_chunks;
+  const int tl = threadIdx.x / kept_chunks, kc = threadIdx.x - tl * kept_chunks;
+  if (tl >= tokens_per_iter) return;
+  const int h = p.kept[kind][kc / p.chunks], c = kc % p.chunks;
+  const int hc = h * p.chunks + c;
   const long long total = static_cast<long long>(per_token) * p.L;
   const uint4* src_k = p.src_k + p.src_stride * slot;
   const uint4* src_v = p.src_v + p.src_stride * slot;
@@ -74,7 +84,6 @@ __global__ void __launch_bounds__(1024) route_block_kernel(const RouteParams p) 
     base = static_cast<long long>(idx) * p.n_blocks * p.L;  // in rows; the rest depends on the token
     spatial = true;
   }
-  if (!dk && !p.copy_mono) return;  // chunks nobody keeps (Sink / Dummy heads of the other blocks) are never loaded
   const int t_stride = gridDim.x * tokens_per_iter;
   for (int t0 = blockIdx.x * tokens_per_iter + tl; t0 < p.L; t0 += t_stride * ROUTE_UNROLL) {
     uint4 kv[ROUTE_UNROLL], vv[ROUTE_UNROLL];

@@ -516,8 +516,25 @@ void fill_route(headcast_ctx* c, RouteParams& r) {
   }
 }
 
-int launch_route(headcast_ctx* c, const RouteParams& r, int n_src, cudaStream_t st) {
-  const int per_token = r.H * r.chunks;  // <= 64 heads * 16 chunks = 1024
+int launch_route(headcast_ctx* c, RouteParams& r, int n_src, cudaStream_t st) {
+  // which heads each kind of source row feeds (see RouteParams::kind)
+  for (int k = 0; k < 4; ++k) {
+    r.n_kept[k] = 0;
+    for (int h = 0; h < r.H; ++h) {
+      const int cl = r.cls[h];
+      const bool keep = r.copy_mono || ((cl == CLS_GLOBAL || cl == CLS_SPATIAL) && r.copy_window) ||
+                        (cl == CLS_SINK && (k == 0 || k == 2)) || (cl == CLS_DUMMY && (k == 1 || k == 2));
+      if (keep) r.kept[k][r.n_kept[k]++] = static_cast<int8_t>(h);
+    }
+  }
+  int max_kept = 0;
+  for (int i = 0; i < n_src; ++i) {
+    const bool s = (i == r.sink_src), d = (i == r.dummy_src);
+    r.kind[i] = static_cast<int8_t>(s && d ? 2 : s ? 0 : d ? 1 : 3);
+    max_kept = std::max<int>(max_kept, r.n_kept[r.kind[i]]);
+  }
+  if (max_kept == 0) return HC_OK;  // nothing to move (e.g. an append when every head is a Sink head)
+  const int per_token = max_kept * r.chunks;  // <= 64 heads * 16 chunks = 1024
   const int tokens_per_iter = std::max(1, 256 / per_token);
   const int threads = tokens_per_iter * per_token;
   const int resident = std::max(1, 2048 / threads);  // blocks per SM
