@@ -390,7 +390,7 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const AttnParams 
           }
         }
         const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
-        // pass 2: p = 2^(s * c - m), row sum in fp32, bf16 pack over the first 32 columns of this thread's logits
+        // pass 2: p = 2^(s * c - m), bf16 pack over the first 32 columns of this thread's logits, row sum in fp32
         const uint64_t c2 = pack_f32x2(p.scale_log2e, p.scale_log2e), m2 = pack_f32x2(-m_use, -m_use);
         uint64_t sum2[2] = {0ull, 0ull};
 #pragma unroll
@@ -414,7 +414,9 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const AttnParams 
               e1 = ex2_approx(x1);
             }
             pk[i] = pack_bf16x2(e0, e1);
-            sum2[i & 1] = add_f32x2(sum2[i & 1], pack_f32x2(e0, e1));
+            // the row sum adds the ROUNDED values: out = sum(p v) / sum(p) is then an exact convex combination of
+            // the values even when the reference lags behind the row maximum and the largest p is not exactly 1
+            sum2[i & 1] = add_f32x2(sum2[i & 1], pack_f32x2(__uint_as_float(pk[i] << 16), __uint_as_float(pk[i] & 0xffff0000u)));
           }
           tmem_st16(p_addr + ch * 16, pk);
         }
