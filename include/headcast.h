@@ -174,6 +174,12 @@ int headcast_plan_schedule(const headcast_config* cfg, const int32_t* labels_hos
                            int32_t dense, int32_t* items_host, int32_t capacity, int32_t* n_items_host,
                            int32_t* cta_first_host);
 
+/* Self-test of the failure path.  Launches one small kernel that waits on a barrier nobody will ever signal; the wait
+ * is bounded like every wait in this library, so after limit_ms (1..1000) the kernel records its give-up in the status
+ * word and returns normally.  The call synchronises `stream` and returns HC_ERR_TIMEOUT - that is the expected
+ * result; the context stays fully usable afterwards.  Nothing faults, traps or hangs. */
+int headcast_selftest_bounded_wait(headcast_ctx* ctx, int32_t limit_ms, void* stream);
+
 /* Synchronises `stream` and reports a device-side status raised by any earlier kernel of this context
  * (HC_ERR_TIMEOUT if a bounded wait expired). */
 int headcast_check(headcast_ctx* ctx, void* stream);

@@ -23,7 +23,7 @@ EXPORTS = ("headcast_default_config", "headcast_create", "headcast_destroy", "he
            "headcast_launch_count", "headcast_attend_flops", "headcast_check", "headcast_last_error",
            "headcast_set_kernel_timing", "headcast_last_attention_kernel_ms", "headcast_set_tracing",
            "headcast_read_trace", "headcast_dense_attend_noalloc", "headcast_noalloc_status",
-           "headcast_noalloc_last_error", "headcast_plan_schedule")
+           "headcast_noalloc_last_error", "headcast_plan_schedule", "headcast_selftest_bounded_wait")
 
 
 class Config(C.Structure):
@@ -76,6 +76,7 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.headcast_read_trace.argtypes = [vp, C.POINTER(C.c_int64), C.c_int32, i32p]
     lib.headcast_dense_attend_noalloc.argtypes = [vp, vp, vp, vp, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_float, vp]
     lib.headcast_noalloc_status.argtypes = [vp]
+    lib.headcast_selftest_bounded_wait.argtypes = [vp, C.c_int32, vp]
     lib.headcast_plan_schedule.argtypes = [C.POINTER(Config), i32p, C.c_int32, C.c_int32, C.c_int32, i32p, C.c_int32, i32p, i32p]
     lib.headcast_noalloc_last_error.argtypes = []
     lib.headcast_noalloc_last_error.restype = C.c_char_p
@@ -265,6 +266,10 @@ class HeadCast:
         rows = np.zeros((max(n.value, 1), 8), dtype=np.int64)
         self._check(self.lib.headcast_read_trace(self._ctx, rows.ctypes.data_as(C.POINTER(C.c_int64)), n.value, C.byref(n)))
         return rows[: n.value]
+
+    def selftest_bounded_wait(self, limit_ms: int = 50) -> int:
+        """Returns the library's status code (HC_ERR_TIMEOUT = -6 is the expected outcome)."""
+        return self.lib.headcast_selftest_bounded_wait(self._ctx, int(limit_ms), _stream())
 
     def check(self) -> None:
         self._check(self.lib.headcast_check(self._ctx, _stream()))

@@ -491,6 +491,21 @@ int run_schedule(headcast_ctx* c, Schedule& s, const void* q, void* out, bool pr
   return HC_OK;
 }
 
+// Self-test of the bounded-wait machinery: one CTA waits on an mbarrier that nobody ever arrives on, gives up after
+// limit_ns, records `code` in the status word and returns normally (no trap, no fault: the context stays usable).
+__global__ void bounded_wait_selftest_kernel(int32_t* status, unsigned long long limit_ns, int code) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 1);
+    abort_flag = 0;
+    fence_mbar_init();
+  }
+  __syncthreads();
+  volatile int* abortp = &abort_flag;
+  mbar_wait_limit(&bar, 0, abortp, status, code, limit_ns);  // every thread waits; the first to expire raises the flag
+}
+
 void fill_route(headcast_ctx* c, RouteParams& r) {
   std::memset(&r, 0, sizeof(r));
   r.mono_k = reinterpret_cast<uint4*>(c->mono_k);
@@ -1085,6 +1100,15 @@ int headcast_plan_schedule(const headcast_config* cfg, const int32_t* labels_hos
     std::memcpy(items_host, s.items.data(), std::min<size_t>(s.items.size(), capacity) * sizeof(WorkItem));
   if (cta_first_host) std::copy(s.cta_first.begin(), s.cta_first.end(), cta_first_host);
   return HC_OK;
+}
+
+int headcast_selftest_bounded_wait(headcast_ctx* c, int32_t limit_ms, void* stream) {
+  if (!c || limit_ms < 1 || limit_ms > 1000) return HC_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  bounded_wait_selftest_kernel<<<1, 64, 0, st>>>(c->status_dev, static_cast<unsigned long long>(limit_ms) * 1000000ull, 99);
+  HC_CUDA(c, cudaGetLastError());
+  ++c->launches;
+  return read_status(c, st);
 }
 
 int headcast_check(headcast_ctx* c, void* stream) {

@@ -52,8 +52,8 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
 #ifndef HC_WAIT_LIMIT_NS
 #define HC_WAIT_LIMIT_NS 2000000000ull
 #endif
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status,
-                                          int code) {
+__device__ __forceinline__ bool mbar_wait_limit(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status,
+                                                int code, uint64_t limit_ns) {
   if (mbar_try_wait(bar, parity)) return true;
   uint64_t t0 = 0;
   for (uint32_t spin = 1;; ++spin) {
@@ -62,13 +62,17 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
       if (*abort_flag) return false;
       uint64_t now = global_timer_ns();
       if (t0 == 0) t0 = now;
-      if (now - t0 > HC_WAIT_LIMIT_NS) {
+      if (now - t0 > limit_ns) {
         *abort_flag = 1;
         atomicCAS(status, 0, code);
         return false;
       }
     }
   }
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status,
+                                          int code) {
+  return mbar_wait_limit(bar, parity, abort_flag, status, code, HC_WAIT_LIMIT_NS);
 }
 
 // generic-proxy writes to shared memory -> visible to the async proxy (TMA, tcgen05.mma operands)

@@ -300,3 +300,18 @@ def test_rollout_sequence_three_layers():
             p.check_cache()
             for step in (0, 3):
                 p.check_attention(dense=False, rows=rows, step=step)
+
+
+def test_an_expired_wait_is_reported_and_the_context_stays_usable():
+    # failure detection without a GPU fault: a kernel waits (bounded) on a barrier nothing signals, gives up after
+    # 50 ms, the host sees HC_ERR_TIMEOUT, and the same context then computes correct attention
+    import time
+    w = synth.tiny()
+    p = Pair(w)
+    p.append(2)
+    t0 = time.perf_counter()
+    assert p.hc.selftest_bounded_wait(50) == -6
+    assert 0.04 < time.perf_counter() - t0 < 5.0
+    assert "bounded wait" in p.hc.lib.headcast_last_error(p.hc._ctx).decode()
+    p.hc.check()  # the status word was cleared by the report
+    p.check_attention(dense=True)
