@@ -266,6 +266,8 @@ def main():
     ap.add_argument("--layers", type=int, default=30, help="rollout: attention layers (one context each)")
     ap.add_argument("--blocks", type=int, default=20, help="rollout: generated blocks after the warm-up")
     ap.add_argument("--impl", default="headcast", choices=["headcast", "reference"])
+    ap.add_argument("--sd-mode", type=int, default=0, choices=[0, 1],
+                    help="1: Sink / Dummy heads keep anchor + current block (Appendix B accounting) instead of one block")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-phases", action="store_true")
     args = ap.parse_args()
@@ -295,7 +297,7 @@ def main():
     flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
     flush = lambda: flush_buf.zero_()
 
-    hc = HeadCast.from_workload(w, keep_monolithic=True)
+    hc = HeadCast.from_workload(w, keep_monolithic=True, sd_mode=args.sd_mode)
     n_extra = 3  # generated blocks fed round-robin once the cache rolls, each with its own 4 denoise-step queries
     kv = [tuple(to_dev(t, torch) for t in synth.make_kv(w, b)) for b in range(w.n_blocks + n_extra)]
     q_fill = to_dev(synth.make_q(w, w.n_blocks - 1, 0), torch)
@@ -456,7 +458,7 @@ def main():
         "dtype": "bf16", "data": "synthetic",
         "config": {"workload": w.name, "heads": H, "head_dim": D, "grid": [w.grid_h, w.grid_w], "block_tokens": L,
                    "kv_tokens": w.n_blocks * L, "head_mix_sink_dummy_spatial_global": [int(sum(1 for v in w.labels if v == c)) for c in range(4)],
-                   "step": "1 attend per step + 1 append per 4 steps", "l2": "flushed between steps (256 MiB memset outside the events)",
+                   "step": "1 attend per step + 1 append per 4 steps", "sd_mode": args.sd_mode, "l2": "flushed between steps (256 MiB memset outside the events)",
                    "parallelism": "replicas only" if world > 1 else "single GPU"},
         "clocks": clocks.summary(),
         "e2e": {"value": e2e, "unit": "ms", "h2d_bytes_per_step": q_bytes + block_bytes // STEPS_PER_BLOCK, "d2h_bytes_per_step": q_bytes},

@@ -83,6 +83,9 @@ typedef struct headcast_config {
   float softmax_scale;      /* 0 selects 1/sqrt(d) */
   int32_t keep_monolithic;  /* nonzero: keep appending to the monolithic cache after the split, so that
                                headcast_full_attend (the dense baseline) stays usable on the same history */
+  int32_t sd_mode;          /* 0: Sink and Dummy heads keep exactly one block (Sec. 4.3, 4.4).  1: the accounting of
+                               Appendix B / C: Sink keeps its anchor block plus the current block, Dummy the previous
+                               plus the current block (2L tokens each) */
 } headcast_config;
 
 typedef struct headcast_ctx headcast_ctx;
@@ -104,6 +107,11 @@ int headcast_destroy(headcast_ctx* ctx);
  * the per-archetype buffers: Sink heads keep their frozen first block, Dummy heads overwrite their single
  * block, Global and Spatial heads slide their window.  Pure byte movement: stored values are bit-identical. */
 int headcast_append(headcast_ctx* ctx, const void* k_new_dev, const void* v_new_dev, void* stream);
+
+/* Per-denoise-step refresh: replaces the K and V of the NEWEST cached block wherever it is kept as the newest block
+ * (monolithic cache, Global / Spatial windows, a Dummy head's current block, a Sink head's current block with
+ * sd_mode 1); no block is evicted and a Sink head's anchor block stays frozen.  Needs at least one cached block. */
+int headcast_overwrite_last(headcast_ctx* ctx, const void* k_new_dev, const void* v_new_dev, void* stream);
 
 /* Dense baseline and warm-up path (Sec. 3.1; "Global Path", Sec. 4.4): every head attends to every cached
  * token of the monolithic cache.  q_dev and out_dev are [L][H][d] bf16.  Needs at least one cached block;

@@ -146,9 +146,12 @@ class CacheModel:
     """List model of the KV cache (Sec. 3.1, 4.3).  ``blocks`` holds (K, V) pairs of
     uint16 [L, H, d] arrays in logical order: index 0 is the sink block, the last is the newest."""
 
-    def __init__(self, n_blocks: int, n_heads: int):
+    def __init__(self, n_blocks: int, n_heads: int, sd_mode: int = 0):
         self.n_blocks = n_blocks
         self.n_heads = n_heads
+        # 0: Sink / Dummy heads keep exactly one block (Sec. 4.3, 4.4); 1: the appendix's accounting (App. B, C):
+        # Sink keeps its anchor block plus the current block, Dummy the previous plus the current block (2L tokens)
+        self.sd_mode = sd_mode
         self.blocks: List[Tuple[np.ndarray, np.ndarray]] = []
         self.labels: Optional[np.ndarray] = None
         self.per_head: Optional[List[List[Tuple[np.ndarray, np.ndarray]]]] = None
@@ -169,9 +172,11 @@ class CacheModel:
             item = (k[:, h, :], v[:, h, :])
             lab = self.labels[h]
             if lab == SINK:
-                pass  # frozen initial block
+                if self.sd_mode == 1:
+                    self.per_head[h] = [self.per_head[h][0], item]  # anchor stays frozen, current block follows
+                # else: frozen initial block
             elif lab == DUMMY:
-                self.per_head[h] = [item]  # rolling overwrite
+                self.per_head[h] = [self.per_head[h][-1], item] if self.sd_mode == 1 else [item]  # rolling overwrite
             else:
                 self._roll(self.per_head[h], item, self.n_blocks)
 
@@ -183,11 +188,25 @@ class CacheModel:
             all_blocks = [(k[:, h, :], v[:, h, :]) for k, v in self.blocks]
             lab = self.labels[h]
             if lab == SINK:
-                self.per_head.append(all_blocks[:1])
+                both = self.sd_mode == 1 and len(all_blocks) > 1
+                self.per_head.append([all_blocks[0], all_blocks[-1]] if both else all_blocks[:1])
             elif lab == DUMMY:
-                self.per_head.append(all_blocks[-1:])
+                self.per_head.append(all_blocks[-2:] if self.sd_mode == 1 else all_blocks[-1:])
             else:
                 self.per_head.append(all_blocks)
+
+    def overwrite_last(self, k: np.ndarray, v: np.ndarray) -> None:
+        """Per-denoise-step refresh: the newest block is replaced wherever it is kept as the newest block (the
+        monolithic cache, the windows, a Dummy head's current block, a Sink head's current block in sd_mode 1).
+        A Sink head's anchor block stays frozen."""
+        self.blocks[-1] = (k, v)
+        if self.per_head is None:
+            return
+        for h in range(self.n_heads):
+            lab = self.labels[h]
+            if lab == SINK and not (self.sd_mode == 1 and len(self.per_head[h]) > 1):
+                continue
+            self.per_head[h][-1] = (k[:, h, :], v[:, h, :])
 
     def head_kv_bits(self, h: int) -> Tuple[np.ndarray, np.ndarray]:
         """Logical content kept for head ``h`` as uint16 [n_tokens, d] (oldest block first)."""

@@ -23,7 +23,7 @@ EXPORTS = ("headcast_default_config", "headcast_create", "headcast_destroy", "he
            "headcast_launch_count", "headcast_attend_flops", "headcast_check", "headcast_last_error",
            "headcast_set_kernel_timing", "headcast_last_attention_kernel_ms", "headcast_set_tracing",
            "headcast_read_trace", "headcast_dense_attend_noalloc", "headcast_noalloc_status",
-           "headcast_noalloc_last_error", "headcast_plan_schedule", "headcast_selftest_bounded_wait")
+           "headcast_noalloc_last_error", "headcast_plan_schedule", "headcast_selftest_bounded_wait", "headcast_overwrite_last")
 
 
 class Config(C.Structure):
@@ -33,7 +33,7 @@ class Config(C.Structure):
                 ("col_edges_host", C.POINTER(C.c_int32)), ("n_col_edges", C.c_int32),
                 ("proxy_radius", C.c_int32), ("theta_sink", C.c_float), ("theta_dummy", C.c_float),
                 ("theta_spatial", C.c_float), ("theta_score", C.c_float), ("gamma", C.c_float),
-                ("softmax_scale", C.c_float), ("keep_monolithic", C.c_int32)]
+                ("softmax_scale", C.c_float), ("keep_monolithic", C.c_int32), ("sd_mode", C.c_int32)]
 
 
 class HeadCastError(RuntimeError):
@@ -58,6 +58,7 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.headcast_destroy.argtypes = [vp]
     lib.headcast_append.argtypes = [vp, vp, vp, vp]
     lib.headcast_full_attend.argtypes = [vp, vp, vp, vp]
+    lib.headcast_overwrite_last.argtypes = [vp, vp, vp, vp]
     lib.headcast_classify.argtypes = [vp, vp, i32p, f32p, vp]
     lib.headcast_set_labels.argtypes = [vp, i32p]
     lib.headcast_get_labels.argtypes = [vp, i32p]
@@ -200,6 +201,9 @@ class HeadCast:
 
     def append(self, k_new, v_new) -> None:
         self._check(self.lib.headcast_append(self._ctx, _ptr(k_new), _ptr(v_new), _stream()))
+
+    def overwrite_last(self, k_new, v_new) -> None:
+        self._check(self.lib.headcast_overwrite_last(self._ctx, _ptr(k_new), _ptr(v_new), _stream()))
 
     def full_attend(self, q, out) -> None:
         self._check(self.lib.headcast_full_attend(self._ctx, _ptr(q), _ptr(out), _stream()))

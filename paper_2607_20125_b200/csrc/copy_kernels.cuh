@@ -20,7 +20,7 @@ struct RouteParams {
   // destinations (any may be null)
   uint4* mono_k;
   uint4* mono_v;
-  uint4* sd_k;  // [N_sink + N_dummy][L][d]
+  uint4* sd_k;  // [N_sink + N_dummy][sd_slots][L][d]
   uint4* sd_v;
   uint4* g_k;   // [N_global][n_blocks * L][d], block slots are a ring
   uint4* g_v;
@@ -33,9 +33,11 @@ struct RouteParams {
   int32_t n_sink;
   int32_t copy_mono, copy_window;
   // blockIdx.y selects the source block: it is read at src + src_stride * slots[y] (stride 0: the caller's block)
-  // and lands in ring slot slots[y]; only source sink_src feeds the Sink heads, only dummy_src the Dummy heads
+  // and lands in ring slot slots[y]; sd_slot_sink[y] / sd_slot_dummy[y] name the block slot of the Sink-Dummy
+  // buffer that source feeds for Sink / Dummy heads (-1: none)
   long long src_stride;    // in 16-byte chunks
-  int32_t sink_src, dummy_src;
+  int32_t sd_slots;        // blocks per head in the Sink-Dummy buffer (1, or 2 with the anchor + current variant)
+  int8_t sd_slot_sink[MAX_BLOCKS], sd_slot_dummy[MAX_BLOCKS];
   int8_t slots[MAX_BLOCKS];
   // threads are laid over the heads somebody keeps: kept[k] lists them for source rows of kind k
   // (0: feeds the Sink heads too, 1: the Dummy heads too, 2: both, 3: neither), n_kept[k] counts them
@@ -70,12 +72,12 @@ __global__ void __launch_bounds__(1024) route_block_kernel(const RouteParams p) 
   uint4 *dk = nullptr, *dv = nullptr;
   long long base = 0;
   bool spatial = false;
-  if (cls == CLS_SINK && src == p.sink_src) {
+  if (cls == CLS_SINK && p.sd_slot_sink[src] >= 0) {
     dk = p.sd_k; dv = p.sd_v;
-    base = static_cast<long long>(idx) * p.L * p.chunks + c;
-  } else if (cls == CLS_DUMMY && src == p.dummy_src) {
+    base = (static_cast<long long>(idx) * p.sd_slots + p.sd_slot_sink[src]) * p.L * p.chunks + c;
+  } else if (cls == CLS_DUMMY && p.sd_slot_dummy[src] >= 0) {
     dk = p.sd_k; dv = p.sd_v;
-    base = static_cast<long long>(p.n_sink + idx) * p.L * p.chunks + c;
+    base = (static_cast<long long>(p.n_sink + idx) * p.sd_slots + p.sd_slot_dummy[src]) * p.L * p.chunks + c;
   } else if (cls == CLS_GLOBAL && p.copy_window) {
     dk = p.g_k; dv = p.g_v;
     base = (static_cast<long long>(idx) * p.n_blocks + slot) * p.L * p.chunks + c;
@@ -134,7 +136,8 @@ struct ExportParams {
   const int32_t* sp_base;
   const int32_t* sp_nc;
   int32_t L, H, chunks, tokens_per_frame, frames_per_block, n_blocks;
-  int32_t layout;      // 0: monolithic [slot][L][H][d]; 1: [head][slot][L][d]; 2: Spatial cell-major; 3: [head][L][d]
+  int32_t layout;      // 0: monolithic [slot][L][H][d]; 1: [head][slot][L][d]; 2: Spatial cell-major; 3: Sink-Dummy [head][sd_slots][L][d]
+  int32_t sd_slots;
   int32_t head;        // original head (layout 0) or index inside the group (others)
   int32_t n_logical;
   int32_t slots[MAX_BLOCKS];  // physical slot of each logical block
@@ -158,7 +161,7 @@ __global__ void __launch_bounds__(256) export_head_kernel(const ExportParams p) 
       s = (static_cast<long long>(p.head) * p.n_blocks * p.L + p.sp_base[pos] +
            static_cast<long long>(slot * p.frames_per_block + f) * p.sp_nc[pos]) * p.chunks + c;
     } else {
-      s = (static_cast<long long>(p.head) * p.L + t) * p.chunks + c;
+      s = ((static_cast<long long>(p.head) * p.sd_slots + slot) * p.L + t) * p.chunks + c;
     }
     if (p.dst_k) p.dst_k[g] = p.src_k[s];
     if (p.dst_v) p.dst_v[g] = p.src_v[s];

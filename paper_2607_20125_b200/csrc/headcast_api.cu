@@ -74,6 +74,9 @@ struct headcast_ctx {
   bool have_labels = false;
   std::vector<int32_t> labels;
   int n_cls[4] = {0, 0, 0, 0};
+  int sd_slots = 1;   // blocks per head in the Sink-Dummy buffer (2 with sd_mode 1)
+  int sd_valid = 0;   // of which hold data
+  int dummy_cur = 0;  // slot holding a Dummy head's newest block
   int8_t cls[MAX_HEADS], idx[MAX_HEADS];
   std::vector<int> row_edges, col_edges;
   std::vector<CellGeom> cells;
@@ -160,7 +163,7 @@ int build_maps(headcast_ctx* c) {
                                  static_cast<uint64_t>(c->H) * c->D, 128);
   }
   if (c->sd_k) {
-    const uint64_t rows = static_cast<uint64_t>(c->n_cls[CLS_SINK] + c->n_cls[CLS_DUMMY]) * c->L;
+    const uint64_t rows = static_cast<uint64_t>(c->n_cls[CLS_SINK] + c->n_cls[CLS_DUMMY]) * c->sd_slots * c->L;
     ok = ok && make_tmap_bf16_2d(&maps[2 * MAP_SD], c->sd_k, c->D, rows, c->D, 128);
     ok = ok && make_tmap_bf16_2d(&maps[2 * MAP_SD + 1], c->sd_v, c->D, rows, c->D, 128);
   }
@@ -369,9 +372,12 @@ void build_headcast_schedule(headcast_ctx* c, Schedule& s) {
     const int cl = c->cls[h], ix = c->idx[h];
     if (cl == CLS_SINK || cl == CLS_DUMMY) {
       const int j = (cl == CLS_SINK) ? ix : c->n_cls[CLS_SINK] + ix;
-      WorkItem w = range_item(h, MAP_SD, 0, static_cast<long long>(j) * c->L, c->L);
+      // the head's blocks are adjacent; with two of them the order does not matter to attention
+      long long row0 = static_cast<long long>(j) * c->sd_slots * c->L;
+      if (cl == CLS_DUMMY && c->sd_valid == 1) row0 += static_cast<long long>(c->dummy_cur) * c->L;
+      WorkItem w = range_item(h, MAP_SD, 0, row0, c->sd_valid * c->L);
       add_query_pairs(protos, w, c->L, w.tiles_per_seg);
-      flops += 4.0 * c->L * static_cast<double>(c->L) * c->D;
+      flops += 4.0 * c->L * static_cast<double>(c->sd_valid) * c->L * c->D;
     } else if (cl == CLS_GLOBAL) {
       WorkItem w = range_item(h, MAP_GLOBAL, 0, ix * win, nf * c->L);
       add_query_pairs(protos, w, c->L, w.tiles_per_seg);
@@ -389,7 +395,7 @@ void build_headcast_schedule(headcast_ctx* c, Schedule& s) {
   }
   s.flops = flops;
   finalize_schedule(c, s, protos, true);
-  s.key_filled = nf;
+  s.key_filled = nf * 4 + c->sd_valid;
 }
 
 int upload_schedule(headcast_ctx* c, Schedule& s, cudaStream_t st) {
@@ -525,6 +531,8 @@ void fill_route(headcast_ctx* c, RouteParams& r) {
   r.frames_per_block = c->F_b;
   r.n_blocks = c->n_blk;
   r.n_sink = c->n_cls[CLS_SINK];
+  r.sd_slots = c->sd_slots;
+  for (int i = 0; i < MAX_BLOCKS; ++i) r.sd_slot_sink[i] = r.sd_slot_dummy[i] = -1;
   for (int h = 0; h < c->H; ++h) {
     r.cls[h] = (c->state == STATE_SPLIT || c->sd_k || c->g_k || c->sp_k) ? c->cls[h] : static_cast<int8_t>(CLS_NONE);
     r.idx[h] = c->idx[h];
@@ -544,7 +552,7 @@ int launch_route(headcast_ctx* c, RouteParams& r, int n_src, cudaStream_t st) {
   }
   int max_kept = 0;
   for (int i = 0; i < n_src; ++i) {
-    const bool s = (i == r.sink_src), d = (i == r.dummy_src);
+    const bool s = r.sd_slot_sink[i] >= 0, d = r.sd_slot_dummy[i] >= 0;
     r.kind[i] = static_cast<int8_t>(s && d ? 2 : s ? 0 : d ? 1 : 3);
     max_kept = std::max<int>(max_kept, r.n_kept[r.kind[i]]);
   }
@@ -587,7 +595,7 @@ static int init_host(headcast_ctx* c, const headcast_config* cfg, std::vector<in
   if (cfg->n_heads < 1 || cfg->n_heads > MAX_HEADS || (cfg->head_dim != 64 && cfg->head_dim != 128) ||
       cfg->grid_h < 1 || cfg->grid_w < 1 || cfg->frames_per_block < 1 || cfg->n_blocks < 2 ||
       cfg->n_blocks > MAX_BLOCKS || cfg->cell_h < 1 || cfg->cell_w < 1 || cfg->proxy_radius < 0 ||
-      !(cfg->softmax_scale >= 0.0f))
+      !(cfg->softmax_scale >= 0.0f) || cfg->sd_mode < 0 || cfg->sd_mode > 1)
     return HC_ERR_INVALID_ARG;
   const long long L = static_cast<long long>(cfg->frames_per_block) * cfg->grid_h * cfg->grid_w;
   if (L * cfg->n_blocks * cfg->n_heads * cfg->head_dim >= (1LL << 40) || L * cfg->n_blocks * cfg->n_heads >= (1LL << 31))
@@ -602,6 +610,7 @@ static int init_host(headcast_ctx* c, const headcast_config* cfg, std::vector<in
   c->L = static_cast<int>(L);
   c->n_blk = cfg->n_blocks;
   c->CH = c->D / 8;
+  c->sd_slots = cfg->sd_mode ? 2 : 1;
   c->scale = cfg->softmax_scale > 0.f ? cfg->softmax_scale : 1.0f / std::sqrt(static_cast<float>(c->D));
   c->row_edges = (cfg->row_edges_host && cfg->n_row_edges > 0)
                      ? std::vector<int>(cfg->row_edges_host, cfg->row_edges_host + cfg->n_row_edges)
@@ -752,6 +761,8 @@ int headcast_append(headcast_ctx* c, const void* k_new, const void* v_new, void*
     next.erase(next.begin() + 1);
     next.push_back(slot);
   }
+  const bool split = c->state == STATE_SPLIT;
+  const int dummy_next = (c->sd_slots == 2) ? (c->dummy_cur ^ 1) : 0;  // the older of a Dummy head's two blocks is replaced
   RouteParams r;
   fill_route(c, r);
   r.src_k = static_cast<const uint4*>(k_new);
@@ -759,13 +770,35 @@ int headcast_append(headcast_ctx* c, const void* k_new, const void* v_new, void*
   r.slots[0] = static_cast<int8_t>(slot);
   r.src_stride = 0;
   r.copy_mono = c->mono_k != nullptr;
-  r.sink_src = -1;  // frozen
-  r.dummy_src = (c->state == STATE_SPLIT) ? 0 : -1;
-  r.copy_window = c->state == STATE_SPLIT;
+  r.sd_slot_sink[0] = static_cast<int8_t>((split && c->sd_slots == 2) ? 1 : -1);  // the anchor block stays frozen
+  r.sd_slot_dummy[0] = static_cast<int8_t>(split ? dummy_next : -1);
+  r.copy_window = split;
   int rc = launch_route(c, r, 1, st);
   if (rc != HC_OK) return rc;
   c->slots.swap(next);
+  if (split) {
+    c->dummy_cur = dummy_next;
+    c->sd_valid = c->sd_slots;
+  }
   return HC_OK;
+}
+
+int headcast_overwrite_last(headcast_ctx* c, const void* k_new, const void* v_new, void* stream) {
+  if (!c) return HC_ERR_INVALID_ARG;
+  if (!aligned16(k_new) || !aligned16(v_new)) return fail(c, HC_ERR_INVALID_ARG, "k_new/v_new must be 16-byte aligned device pointers");
+  if (c->slots.empty()) return fail(c, HC_ERR_STATE, "the cache is empty");
+  const bool split = c->state == STATE_SPLIT;
+  RouteParams r;
+  fill_route(c, r);
+  r.src_k = static_cast<const uint4*>(k_new);
+  r.src_v = static_cast<const uint4*>(v_new);
+  r.slots[0] = static_cast<int8_t>(c->slots.back());
+  r.src_stride = 0;
+  r.copy_mono = c->mono_k != nullptr;
+  r.sd_slot_sink[0] = static_cast<int8_t>((split && c->sd_slots == 2 && c->sd_valid == 2) ? 1 : -1);
+  r.sd_slot_dummy[0] = static_cast<int8_t>(split ? c->dummy_cur : -1);
+  r.copy_window = split;
+  return launch_route(c, r, 1, static_cast<cudaStream_t>(stream));
 }
 
 int headcast_full_attend(headcast_ctx* c, const void* q, void* out, void* stream) {
@@ -906,7 +939,7 @@ int headcast_split_cache(headcast_ctx* c, void* stream) {
   assign_classes(c);
   // carve the three buffers out of the arena reserved (and zeroed) at create: no allocation on this path
   const int n_sd = c->n_cls[CLS_SINK] + c->n_cls[CLS_DUMMY];
-  const size_t sd_elems = static_cast<size_t>(n_sd) * c->L * c->D;
+  const size_t sd_elems = static_cast<size_t>(n_sd) * c->sd_slots * c->L * c->D;
   const size_t g_elems = cache_elems(c, c->n_cls[CLS_GLOBAL]);
   const size_t sp_elems = cache_elems(c, c->n_cls[CLS_SPATIAL]);
   c->sd_k = sd_elems ? c->arena_k : nullptr;
@@ -924,8 +957,19 @@ int headcast_split_cache(headcast_ctx* c, void* stream) {
     r.src_stride = static_cast<long long>(c->L) * c->H * c->CH;
     for (size_t i = 0; i < c->slots.size(); ++i) r.slots[i] = static_cast<int8_t>(c->slots[i]);
     r.copy_mono = 0;
-    r.sink_src = 0;
-    r.dummy_src = static_cast<int32_t>(c->slots.size()) - 1;
+    const int n = static_cast<int>(c->slots.size());
+    r.sd_slot_sink[0] = 0;  // the first block is the Sink heads' anchor
+    if (c->sd_slots == 2 && n >= 2) {
+      r.sd_slot_sink[n - 1] = 1;   // anchor + current block
+      r.sd_slot_dummy[n - 2] = 0;  // previous + current block
+      r.sd_slot_dummy[n - 1] = 1;
+      c->dummy_cur = 1;
+      c->sd_valid = 2;
+    } else {
+      r.sd_slot_dummy[n - 1] = 0;
+      c->dummy_cur = 0;
+      c->sd_valid = 1;
+    }
     r.copy_window = 1;
     int rc = launch_route(c, r, static_cast<int>(c->slots.size()), st);
     if (rc != HC_OK) return rc;
@@ -945,7 +989,7 @@ int headcast_attend(headcast_ctx* c, const void* q, void* out, void* stream) {
   if (!c) return HC_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(out)) return fail(c, HC_ERR_INVALID_ARG, "q/out must be 16-byte aligned device pointers");
   if (c->state != STATE_SPLIT) return fail(c, HC_ERR_STATE, "head-specific attention needs the split cache");
-  if (c->sched_hc.key_filled != n_filled(c)) build_headcast_schedule(c, c->sched_hc);
+  if (c->sched_hc.key_filled != n_filled(c) * 4 + c->sd_valid) build_headcast_schedule(c, c->sched_hc);
   return run_schedule(c, c->sched_hc, q, out, false, static_cast<cudaStream_t>(stream));
 }
 
@@ -964,6 +1008,7 @@ int headcast_export_cache(headcast_ctx* c, int32_t head, void* k_out, void* v_ou
   e.tokens_per_frame = c->T_f;
   e.frames_per_block = c->F_b;
   e.n_blocks = c->n_blk;
+  e.sd_slots = c->sd_slots;
   const int cl = (c->state == STATE_SPLIT) ? c->cls[head] : CLS_NONE;
   if (cl == CLS_NONE) {
     e.layout = 0; e.head = head; e.src_k = reinterpret_cast<const uint4*>(c->mono_k); e.src_v = reinterpret_cast<const uint4*>(c->mono_v);
@@ -976,8 +1021,16 @@ int headcast_export_cache(headcast_ctx* c, int32_t head, void* k_out, void* v_ou
     e.src_k = reinterpret_cast<const uint4*>(c->sd_k); e.src_v = reinterpret_cast<const uint4*>(c->sd_v);
   }
   if (e.layout == 3) {
-    e.n_logical = c->slots.empty() ? 0 : 1;
-    e.slots[0] = 0;
+    e.n_logical = c->sd_valid;
+    if (cl == CLS_SINK) {
+      e.slots[0] = 0;
+      e.slots[1] = 1;
+    } else if (c->sd_valid == 2) {
+      e.slots[0] = c->dummy_cur ^ 1;  // previous block first
+      e.slots[1] = c->dummy_cur;
+    } else {
+      e.slots[0] = c->dummy_cur;
+    }
   } else {
     e.n_logical = n_filled(c);
     for (int i = 0; i < e.n_logical; ++i) e.slots[i] = c->slots[i];
@@ -1005,7 +1058,8 @@ double headcast_attend_flops(const headcast_ctx* c, int32_t dense) {
   for (const CellGeom& g : c->cells) cell_sq += static_cast<double>(g.ch * g.cw) * (g.ch * g.cw);
   double f = 0.0;
   for (int h = 0; h < c->H; ++h) {
-    if (c->labels[h] == HC_SINK || c->labels[h] == HC_DUMMY) f += 4.0 * c->L * static_cast<double>(c->L) * c->D;
+    if (c->labels[h] == HC_SINK || c->labels[h] == HC_DUMMY)
+      f += 4.0 * c->L * static_cast<double>(c->state == STATE_SPLIT ? c->sd_valid : std::min(c->sd_slots, nf)) * c->L * c->D;
     else if (c->labels[h] == HC_GLOBAL) f += 4.0 * c->L * static_cast<double>(nf) * c->L * c->D;
     else f += 4.0 * c->F_b * static_cast<double>(nf) * c->F_b * cell_sq * c->D;
   }
@@ -1092,6 +1146,8 @@ int headcast_plan_schedule(const headcast_config* cfg, const int32_t* labels_hos
       if (labels_host[h] < 0 || labels_host[h] > 3) return HC_ERR_INVALID_ARG;
     c.labels.assign(labels_host, labels_host + c.H);
     assign_classes(&c);
+    c.sd_valid = std::min(c.sd_slots, n_filled);
+    c.dummy_cur = c.sd_valid - 1;
     build_headcast_schedule(&c, s);
   }
   *n_items_host = static_cast<int32_t>(s.items.size());

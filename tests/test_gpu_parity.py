@@ -36,7 +36,7 @@ class Pair:
         from paper_2607_20125_b200.binding import HeadCast
         self.w = w
         self.hc = HeadCast.from_workload(w, keep_monolithic=keep_monolithic, **kw)
-        self.cache = orc.CacheModel(w.n_blocks, w.n_heads)
+        self.cache = orc.CacheModel(w.n_blocks, w.n_heads, sd_mode=kw.get("sd_mode", 0))
         self.geom = geometry(w, row_edges=kw.get("row_edges"), col_edges=kw.get("col_edges"))
         self.next_block = 0
 
@@ -46,6 +46,12 @@ class Pair:
             self.hc.append(to_dev(k), to_dev(v))
             self.cache.append(k, v)
             self.next_block += 1
+
+    def overwrite_last(self, seed_block):
+        """Per-denoise-step refresh of the newest block with fresh seeded K/V."""
+        k, v = synth.make_kv(self.w, 1000 + seed_block)
+        self.hc.overwrite_last(to_dev(k), to_dev(v))
+        self.cache.overwrite_last(k, v)
 
     def check_cache(self):
         for h in range(self.w.n_heads):
@@ -314,4 +320,48 @@ def test_an_expired_wait_is_reported_and_the_context_stays_usable():
     assert 0.04 < time.perf_counter() - t0 < 5.0
     assert "bounded wait" in p.hc.lib.headcast_last_error(p.hc._ctx).decode()
     p.hc.check()  # the status word was cleared by the report
+    p.check_attention(dense=True)
+
+
+@pytest.mark.parametrize("fill", [1, 2, 4])
+def test_anchor_plus_current_variant_of_sink_and_dummy(fill):
+    # Appendix B / C accounting: Sink = anchor + current block, Dummy = previous + current block; split with 1, 2 or
+    # all 4 blocks cached, then appends that roll the window, with a per-step refresh of the current block in between
+    w = synth.small()
+    p = Pair(w, sd_mode=1)
+    p.append(fill)
+    p.hc.set_labels(w.labels)
+    p.hc.split_cache()
+    p.cache.split(w.labels)
+    p.check_cache()
+    p.check_attention(dense=False)
+    for i in range(4):
+        p.append()
+        p.check_cache()
+        p.check_attention(dense=False, step=i)
+        p.overwrite_last(i)
+        p.check_cache()
+        p.check_attention(dense=False, step=i)
+    p.check_attention(dense=True)
+    L = w.block_tokens
+    assert abs(p.hc.attend_flops(False) - orc.attend_flops(p.geom, w.labels, 4, w.head_dim)
+               - 2 * 4.0 * L * L * w.head_dim) < 1.0  # the 2 Sink/Dummy heads read one more block each
+
+
+def test_refresh_of_the_current_block_in_one_block_mode():
+    w = synth.small()
+    p = Pair(w)
+    p.append(2)
+    p.overwrite_last(0)  # before the split: monolithic cache only
+    p.check_cache()
+    p.check_attention(dense=True)
+    p.hc.set_labels(w.labels)
+    p.hc.split_cache()
+    p.cache.split(w.labels)
+    for i in range(3):
+        p.overwrite_last(1 + i)
+        p.check_cache()
+        p.check_attention(dense=False, step=i)
+        p.append()
+    p.check_cache()
     p.check_attention(dense=True)

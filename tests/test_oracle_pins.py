@@ -393,3 +393,63 @@ def test_generator_is_deterministic_and_bf16_rounding_is_rne():
     assert orc.widen_bf16(np.array([0x3F80, 0xC020], np.uint16)).tolist() == [1.0, -2.5]
     rows = synth.sample_rows(synth.wan("480p"))
     assert rows.min() >= 0 and rows.max() < 4680 and np.all(np.diff(rows) > 0) and rows.size >= 256
+
+
+# ---- appendix variant: Sink / Dummy keep two blocks (App. B, C) ---------------------------
+
+
+def test_two_block_variant_of_sink_and_dummy():
+    rng = np.random.default_rng(21)
+    geom = orc.Geometry.make(4, 6, 3, 2, 3)
+    L, H, d = geom.block_tokens, 3, 16
+    blocks = [(rand_bits(rng, (L, H, d)), rand_bits(rng, (L, H, d))) for _ in range(7)]
+    q = rand_bits(rng, (L, H, d), 2.0)
+    cache = orc.CacheModel(4, H, sd_mode=1)
+    for b in blocks[:3]:
+        cache.append(*b)
+    cache.split([orc.SINK, orc.DUMMY, orc.GLOBAL])
+
+    def ids(h):
+        kb = cache.head_kv_bits(h)[0]
+        return [next(i for i, b in enumerate(blocks) if np.array_equal(b[0][:, h], kb[j * L:(j + 1) * L])) for j in range(kb.shape[0] // L)]
+
+    assert ids(0) == [0, 2] and ids(1) == [1, 2] and ids(2) == [0, 1, 2]
+    for n in range(3, 6):
+        cache.append(*blocks[n])
+        assert ids(0) == [0, n] and ids(1) == [n - 1, n]
+    # attention of a Sink head = dense attention over {anchor, current}; of a Dummy head over {previous, current}
+    two = orc.CacheModel(4, H)
+    two.append(*blocks[0]); two.append(*blocks[5])
+    prev = orc.CacheModel(4, H)
+    prev.append(*blocks[4]); prev.append(*blocks[5])
+    o = orc.attend(q, cache, geom)
+    assert np.array_equal(o[:, 0], orc.full_attend(q, two)[0][:, 0])
+    assert np.array_equal(o[:, 1], orc.full_attend(q, prev)[0][:, 1])
+    # per-denoise-step refresh replaces the current block, never the Sink anchor
+    cache.overwrite_last(*blocks[6])
+    assert ids(0) == [0, 6] and ids(1) == [4, 6] and ids(2)[-1] == 6 and len(ids(2)) == 4
+    # one cached block: anchor and current coincide
+    one = orc.CacheModel(4, H, sd_mode=1)
+    one.append(*blocks[0])
+    one.split([orc.SINK, orc.DUMMY, orc.GLOBAL])
+    assert one.head_kv_bits(0)[0].shape[0] == L and one.head_kv_bits(1)[0].shape[0] == L
+    one.append(*blocks[1])
+    assert one.head_kv_bits(0)[0].shape[0] == 2 * L and one.head_kv_bits(1)[0].shape[0] == 2 * L
+    # memory: the appendix's formula with W = 8 and 2 kept blocks
+    g = golden()
+    sd, tot = g["kv_sink_dummy_share"]
+    assert abs(orc.kv_reduction(sd, tot, 8, 2) - (sd / tot) * 0.75) < 1e-15
+
+
+def test_one_block_mode_refresh_leaves_the_sink_frozen():
+    rng = np.random.default_rng(22)
+    L, H, d = 6, 3, 4
+    blocks = [(rand_bits(rng, (L, H, d)), rand_bits(rng, (L, H, d))) for _ in range(4)]
+    cache = orc.CacheModel(3, H)
+    cache.append(*blocks[0]); cache.append(*blocks[1])
+    cache.split([orc.SINK, orc.DUMMY, orc.SPATIAL])
+    cache.overwrite_last(*blocks[3])
+    assert np.array_equal(cache.head_kv_bits(0)[0], blocks[0][0][:, 0])
+    assert np.array_equal(cache.head_kv_bits(1)[0], blocks[3][0][:, 1])
+    assert np.array_equal(cache.head_kv_bits(2)[0][L:], blocks[3][0][:, 2])
+    assert np.array_equal(cache.mono_kv_bits(0)[0][L:], blocks[3][0][:, 0])
