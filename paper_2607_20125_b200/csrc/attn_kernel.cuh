@@ -106,19 +106,32 @@ __device__ __forceinline__ int cell_query_token(const CellGeom& g, int p, int to
   return f * tokens_per_frame + (g.y0 + dy) * grid_w + g.x0 + dx;
 }
 
-// Sets the logits of keys a query row must not see to -inf: columns >= n_valid (ragged tail of a segment) and,
-// for the Spatial proxy, keys outside the (2r+1)^2 neighbourhood of the query's grid position (qy, qx); tok0 is
-// the in-frame token index of column 0.
+// Which of 32 consecutive keys a query row may see, as a bit mask: columns >= n_valid (ragged tail of a segment) are
+// never seen; for the Spatial proxy neither are keys outside the (2r+1)^2 neighbourhood of the query's grid position
+// (qy, qx).  tok0 is the in-frame token index of column 0.  The neighbourhood is at most 2r+1 runs of consecutive
+// tokens (one per grid row), so the mask costs a few integer operations per row of the neighbourhood, not per key.
 template <bool PROXY>
-__device__ __forceinline__ void mask_logits(uint32_t (&sv)[32], int n_valid, int tok0, int qy, int qx, int radius, int grid_w) {
+__device__ __forceinline__ uint32_t visible_keys(int n_valid, int tok0, int qy, int qx, int radius, int grid_w) {
+  uint32_t tail = (n_valid >= 32) ? 0xffffffffu : (n_valid <= 0 ? 0u : (0xffffffffu >> (32 - n_valid)));
+  if (!PROXY) return tail;
+  uint32_t allow = 0;
+  const int lo_x = max(qx - radius, 0), hi_x = min(qx + radius, grid_w - 1);
+#pragma unroll 1
+  for (int ky = max(qy - radius, 0); ky <= qy + radius; ++ky) {
+    const int a = max(ky * grid_w + lo_x - tok0, 0), b = min(ky * grid_w + hi_x - tok0, 31);  // inclusive column range
+    if (a <= b) allow |= (0xffffffffu >> (31 - b + a)) << a;
+  }
+  return allow & tail;
+}
+
+// Sets the logits of the keys a row must not see to -inf.  Outside the proxy only the ragged tail of a segment is
+// hidden, which is the same for all rows: a comparison per column, skipped for full chunks.
+template <bool PROXY>
+__device__ __forceinline__ void apply_visible(uint32_t (&sv)[32], uint32_t visible, int n_valid) {
   if (PROXY) {
-    int ky = tok0 / grid_w, kx = tok0 - ky * grid_w;
 #pragma unroll
-    for (int i = 0; i < 32; ++i) {
-      const bool a = (i < n_valid) && (abs(ky - qy) <= radius) && (abs(kx - qx) <= radius);
-      if (!a) sv[i] = 0xff800000u;
-      if (++kx == grid_w) { kx = 0; ++ky; }
-    }
+    for (int i = 0; i < 32; ++i)
+      if (!((visible >> i) & 1u)) sv[i] = 0xff800000u;
   } else if (n_valid < 32) {
 #pragma unroll
     for (int i = 0; i < 32; ++i)
@@ -349,10 +362,12 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const AttnParams 
           float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
           for (int ch = 0; ch < 2; ++ch) {
+            const uint32_t visible = PROXY ? visible_keys<PROXY>(n_valid - ch * 32, tok0 + ch * 32, qy, qx, p.radius, p.grid_w) : 0u;
+            if (PROXY && __all_sync(0xffffffffu, visible == 0u)) continue;  // no row of this warp sees any of these keys
             uint32_t sv[32];
             tmem_ld32(s_addr + ch * 32, sv);
             tmem_wait_ld();
-            mask_logits<PROXY>(sv, n_valid - ch * 32, tok0 + ch * 32, qy, qx, p.radius, p.grid_w);
+            apply_visible<PROXY>(sv, visible, n_valid - ch * 32);
 #pragma unroll
             for (int i = 0; i < 32; i += 8) {
               mx4[0] = max3(mx4[0], __uint_as_float(sv[i]), __uint_as_float(sv[i + 1]));
@@ -395,11 +410,19 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const AttnParams 
         uint64_t sum2[2] = {0ull, 0ull};
 #pragma unroll
         for (int ch = 0; ch < 2; ++ch) {
+          const uint32_t visible = PROXY ? visible_keys<PROXY>(n_valid - ch * 32, tok0 + ch * 32, qy, qx, p.radius, p.grid_w) : 0u;
+          uint32_t pk[16];
+          if (PROXY && __all_sync(0xffffffffu, visible == 0u)) {
+            // nothing to exponentiate: P = 0 for these keys (the product still reads them)
+#pragma unroll
+            for (int i = 0; i < 16; ++i) pk[i] = 0u;
+            tmem_st16(p_addr + ch * 16, pk);
+            continue;
+          }
           uint32_t sv[32];
           tmem_ld32(s_addr + ch * 32, sv);
           tmem_wait_ld();
-          mask_logits<PROXY>(sv, n_valid - ch * 32, tok0 + ch * 32, qy, qx, p.radius, p.grid_w);
-          uint32_t pk[16];
+          apply_visible<PROXY>(sv, visible, n_valid - ch * 32);
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
             const uint64_t x2 = fma_f32x2(pack_f32x2(__uint_as_float(sv[2 * i]), __uint_as_float(sv[2 * i + 1])), c2, m2);
