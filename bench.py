@@ -199,7 +199,10 @@ def run_rollout(args):
     qs = [torch.randn((L, H, D), device="cuda", generator=g).bfloat16() for _ in range(STEPS_PER_BLOCK)]
     out = torch.empty_like(qs[0])
     layers = [HeadCast.from_workload(synth.wan("720p", layer=l), keep_monolithic=True) for l in range(args.layers)]
-    mixes = [synth.wan("720p", layer=l).labels for l in range(args.layers)]
+    mixes = (synth.reported_mixes("720p", args.layers) if args.mix == "reported"
+             else [synth.wan("720p", layer=l).labels for l in range(args.layers)])
+    if args.ablation != "full":
+        mixes = [synth.ablation_labels(m)[args.ablation] for m in mixes]
     ev = lambda: torch.cuda.Event(enable_timing=True)
     t = {}
     a, b = ev(), ev()
@@ -248,7 +251,9 @@ def run_rollout(args):
         "metric": "headcast_rollout_attention_ms_per_block_step_all_layers", "value": per_step, "unit": "ms", "n_gpus": 1,
         "steps": n_steps, "warmup": 0, "ms_per_step": per_step, "higher_is_better": False, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic (seeded N(0,1) drawn on the device, shared by the layers)",
-        "config": {"workload": "rollout-720p", "layers": args.layers, "blocks": args.blocks, "steps_per_block": STEPS_PER_BLOCK,
+        "config": {"workload": "rollout-720p", "head_mix": args.mix, "ablation": args.ablation,
+                   "head_counts_sink_dummy_spatial_global": [int(sum(1 for m in mixes for v in m if v == c)) for c in range(4)],
+                   "layers": args.layers, "blocks": args.blocks, "steps_per_block": STEPS_PER_BLOCK,
                    "heads": H, "head_dim": D, "grid": [base.grid_h, base.grid_w], "l2": "working set of 30 layers (48 GB) exceeds L2"},
         "gpu_launches": int(launches),
         "rollout": {**t, "speedup_vs_dense": t["dense_ms"] / t["headcast_ms"],
@@ -268,6 +273,12 @@ def main():
     ap.add_argument("--impl", default="headcast", choices=["headcast", "reference"])
     ap.add_argument("--sd-mode", type=int, default=0, choices=[0, 1],
                     help="1: Sink / Dummy heads keep anchor + current block (Appendix B accounting) instead of one block")
+    ap.add_argument("--mix", default="default", choices=["default", "reported"],
+                    help="rollout: 2/3/4/3 heads per layer, or the 360-head distribution the paper reports for LongLive at 720P")
+    ap.add_argument("--ablation", default="full", choices=["full", "all_global", "spatial_only", "sink_dummy_only"],
+                    help="rollout: which archetypes stay sparse (the paper's archetype ablation); the rest become Global")
+    ap.add_argument("--ablations", action="store_true",
+                    help="single layer: also time headcast_attend for the label sets of the paper's archetype ablation")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-phases", action="store_true")
     args = ap.parse_args()
@@ -420,11 +431,33 @@ def main():
         phases["speedup_vs_dense"] = phases["dense_full_attend_ms"] / attend_ms
         phases["ideal_speedup_by_flops"] = hc.attend_flops(True) / flops
 
-    # ---- end to end through the same calls with host buffers (pinned), copies inside the timed region
+    if args.ablations:
+        # the paper's archetype ablation, attention only: a fresh context per label set, same cache content
+        abl = {}
+        for name, lab in synth.ablation_labels(w.labels).items():
+            h2 = HeadCast.from_workload(w, keep_monolithic=False, sd_mode=args.sd_mode)
+            for blk in range(w.n_blocks):
+                h2.append(*kv[blk])
+            h2.set_labels(lab)
+            h2.split_cache()
+            h2.set_kernel_timing(True)
+            for _ in range(3):
+                h2.attend(q_extra[0][0], out)
+            abl[name + "_ms"] = timed(torch, lambda: h2.attend(q_extra[0][0], out), flush, 10)
+            abl[name + "_gflop"] = h2.attend_flops(False) / 1e9
+            h2.check()
+            h2.destroy()
+        for name in ("spatial_only", "sink_dummy_only", "full"):
+            abl[name + "_speedup"] = abl["all_global_ms"] / abl[name + "_ms"]
+        abl["paper_whole_model_speedups_720p"] = {"spatial_only": 1.19, "sink_dummy_only": 1.04, "full": 1.31}
+        phases["ablation"] = abl
+
+    # ---- end to end: the host-buffer entry points of the C ABI (pinned host tensors), every copy inside the timed
+    # region: headcast_append_host every 4th step, headcast_attend_host (query columns in, outputs out, overlapped
+    # with the kernels group by group), stream synchronised before the clock stops
     host_q = [q.cpu().pin_memory() for q in q_extra[0]]
     host_kv = [(k.cpu().pin_memory(), v.cpu().pin_memory()) for k, v in kv[w.n_blocks:w.n_blocks + 2]]
     host_out = torch.empty_like(host_q[0]).pin_memory()
-    dq, dk, dv = torch.empty_like(q_fill), torch.empty_like(kv[0][0]), torch.empty_like(kv[0][1])
     e2e_steps = min(args.steps, 40)
     e2e_ms = []
     for i in range(-3, e2e_steps):
@@ -432,16 +465,13 @@ def main():
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a.record()
         if i % STEPS_PER_BLOCK == 0:
-            dk.copy_(host_kv[(i // STEPS_PER_BLOCK) % 2][0], non_blocking=True)
-            dv.copy_(host_kv[(i // STEPS_PER_BLOCK) % 2][1], non_blocking=True)
-            hc.append(dk, dv)
-        dq.copy_(host_q[i % STEPS_PER_BLOCK], non_blocking=True)
-        hc.attend(dq, out)
-        host_out.copy_(out, non_blocking=True)
+            hc.append_host(*host_kv[(i // STEPS_PER_BLOCK) % 2])
+        hc.attend_host(host_q[i % STEPS_PER_BLOCK], host_out)
         b.record()
         b.synchronize()
         if i >= 0:
             e2e_ms.append(a.elapsed_time(b))
+    hc.check()
     e2e = float(np.sum(e2e_ms)) / e2e_steps
     if dist is not None:
         tt = torch.tensor([e2e], device="cuda", dtype=torch.float64)

@@ -153,6 +153,19 @@ int headcast_n_filled(const headcast_ctx* ctx);
 /* Number of kernels this context has launched so far (bookkeeping for benchmarks). */
 int64_t headcast_launch_count(const headcast_ctx* ctx);
 
+/* The same two steps for callers whose tensors live in HOST memory (the paper's pipeline keeps them on the GPU; this
+ * is for measuring, or serving, the path end to end across PCIe).  k_host/v_host/q_host/out_host: host pointers to
+ * [L][H][d] bf16; pinned memory lets the copies overlap the kernels, pageable memory works but serialises.
+ * headcast_append_host copies the block into device staging owned by the context and appends it.
+ * headcast_attend_host splits the call by archetype group (Global, Spatial, Sink + Dummy heads): each group's query
+ * columns are copied in, attended (Sec. 4.4, as headcast_attend) and its output columns copied out, on two copy
+ * streams of the context, so that transfers in both directions overlap the attention of the other groups.  Both
+ * return once everything is enqueued; out_host is complete when work enqueued on `stream` after the call runs (e.g.
+ * after synchronising `stream`).  q_host must stay unchanged and out_host untouched until then.  Staging buffers,
+ * streams and events are created on the first call.  Errors as headcast_attend / headcast_append. */
+int headcast_append_host(headcast_ctx* ctx, const void* k_host, const void* v_host, void* stream);
+int headcast_attend_host(headcast_ctx* ctx, const void* q_host, void* out_host, void* stream);
+
 /* Algorithmic FLOPs (4 * L_q * L_k * d per head, Appendix B) of the next headcast_attend (dense = 0) or
  * headcast_full_attend (dense = 1) with the current cache fill and labels. */
 double headcast_attend_flops(const headcast_ctx* ctx, int32_t dense);

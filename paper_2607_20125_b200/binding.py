@@ -23,7 +23,8 @@ EXPORTS = ("headcast_default_config", "headcast_create", "headcast_destroy", "he
            "headcast_launch_count", "headcast_attend_flops", "headcast_check", "headcast_last_error",
            "headcast_set_kernel_timing", "headcast_last_attention_kernel_ms", "headcast_set_tracing",
            "headcast_read_trace", "headcast_dense_attend_noalloc", "headcast_noalloc_status",
-           "headcast_noalloc_last_error", "headcast_plan_schedule", "headcast_selftest_bounded_wait", "headcast_overwrite_last")
+           "headcast_noalloc_last_error", "headcast_plan_schedule", "headcast_selftest_bounded_wait", "headcast_overwrite_last",
+           "headcast_append_host", "headcast_attend_host")
 
 
 class Config(C.Structure):
@@ -64,6 +65,8 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.headcast_get_labels.argtypes = [vp, i32p]
     lib.headcast_split_cache.argtypes = [vp, vp]
     lib.headcast_attend.argtypes = [vp, vp, vp, vp]
+    lib.headcast_append_host.argtypes = [vp, vp, vp, vp]
+    lib.headcast_attend_host.argtypes = [vp, vp, vp, vp]
     lib.headcast_export_cache.argtypes = [vp, C.c_int32, vp, vp, i32p, vp]
     lib.headcast_n_filled.argtypes = [vp]
     lib.headcast_launch_count.argtypes = [vp]
@@ -103,6 +106,11 @@ def _stream() -> int:
 
 def _ptr(t) -> int:
     assert t.is_cuda and t.is_contiguous(), "tensors handed to the library must be contiguous CUDA tensors"
+    return t.data_ptr()
+
+
+def _host_ptr(t) -> int:
+    assert (not t.is_cuda) and t.is_contiguous(), "host entry points take contiguous CPU tensors"
     return t.data_ptr()
 
 
@@ -230,6 +238,14 @@ class HeadCast:
 
     def attend(self, q, out) -> None:
         self._check(self.lib.headcast_attend(self._ctx, _ptr(q), _ptr(out), _stream()))
+
+    def append_host(self, k_host, v_host) -> None:
+        """k_host / v_host: CPU tensors (pinned for overlap) of shape [L, H, d], bf16."""
+        self._check(self.lib.headcast_append_host(self._ctx, _host_ptr(k_host), _host_ptr(v_host), _stream()))
+
+    def attend_host(self, q_host, out_host) -> None:
+        """q_host / out_host: CPU tensors (pinned for overlap); out_host is complete after the stream is synchronised."""
+        self._check(self.lib.headcast_attend_host(self._ctx, _host_ptr(q_host), _host_ptr(out_host), _stream()))
 
     def export_cache(self, head: int):
         """Returns (K, V) uint16 CPU arrays [n_tokens, d] of what the cache keeps for ``head``."""

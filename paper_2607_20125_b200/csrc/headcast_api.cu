@@ -91,6 +91,10 @@ struct headcast_ctx {
   int32_t* status_dev = nullptr;
 
   Schedule sched_dense, sched_hc, sched_cls, sched_proxy;
+  Schedule sched_group[3];  // headcast_attend_host: Global / Spatial / Sink+Dummy heads on their own
+  DevBuf<__nv_bfloat16> stage_q, stage_out, stage_k, stage_v;  // device copies of host tensors
+  cudaStream_t copy_in = nullptr, copy_out = nullptr;
+  cudaEvent_t ev_host[8] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
   DevBuf<float> part_o;
   DevBuf<float2> part_ml;
   DevBuf<float> cls_o, cls_lse, cls_tok, cls_scores;
@@ -363,13 +367,15 @@ void build_dense_schedule(headcast_ctx* c, Schedule& s, int out_mode, bool allow
   s.key_filled = n_filled(c);
 }
 
-void build_headcast_schedule(headcast_ctx* c, Schedule& s) {
+// group < 0: every head; 0: Global heads only; 1: Spatial; 2: Sink and Dummy
+void build_headcast_schedule(headcast_ctx* c, Schedule& s, int group = -1) {
   std::vector<Proto> protos;
   const int nf = n_filled(c);
   const long long win = static_cast<long long>(c->n_blk) * c->L;
   double flops = 0.0;
   for (int h = 0; h < c->H; ++h) {
     const int cl = c->cls[h], ix = c->idx[h];
+    if (group >= 0 && group != (cl == CLS_GLOBAL ? 0 : cl == CLS_SPATIAL ? 1 : 2)) continue;
     if (cl == CLS_SINK || cl == CLS_DUMMY) {
       const int j = (cl == CLS_SINK) ? ix : c->n_cls[CLS_SINK] + ix;
       // the head's blocks are adjacent; with two of them the order does not matter to attention
@@ -732,6 +738,15 @@ int headcast_destroy(headcast_ctx* c) {
   c->sched_hc.release();
   c->sched_cls.release();
   c->sched_proxy.release();
+  for (Schedule& g : c->sched_group) g.release();
+  c->stage_q.release();
+  c->stage_out.release();
+  c->stage_k.release();
+  c->stage_v.release();
+  if (c->copy_in) cudaStreamDestroy(c->copy_in);
+  if (c->copy_out) cudaStreamDestroy(c->copy_out);
+  for (cudaEvent_t e : c->ev_host)
+    if (e) cudaEventDestroy(e);
   c->part_o.release();
   c->part_ml.release();
   c->trace_dev.release();
@@ -991,6 +1006,84 @@ int headcast_attend(headcast_ctx* c, const void* q, void* out, void* stream) {
   if (c->state != STATE_SPLIT) return fail(c, HC_ERR_STATE, "head-specific attention needs the split cache");
   if (c->sched_hc.key_filled != n_filled(c) * 4 + c->sd_valid) build_headcast_schedule(c, c->sched_hc);
   return run_schedule(c, c->sched_hc, q, out, false, static_cast<cudaStream_t>(stream));
+}
+
+namespace {
+
+int init_host_path(headcast_ctx* c) {
+  if (!c->copy_in) HC_CUDA(c, cudaStreamCreateWithFlags(&c->copy_in, cudaStreamNonBlocking));
+  if (!c->copy_out) HC_CUDA(c, cudaStreamCreateWithFlags(&c->copy_out, cudaStreamNonBlocking));
+  for (cudaEvent_t& e : c->ev_host)
+    if (!e) HC_CUDA(c, cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+  return HC_OK;
+}
+
+}  // namespace
+
+int headcast_append_host(headcast_ctx* c, const void* k_host, const void* v_host, void* stream) {
+  if (!c || !k_host || !v_host) return HC_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t elems = static_cast<size_t>(c->L) * c->H * c->D;
+  HC_CUDA(c, c->stage_k.reserve(elems));
+  HC_CUDA(c, c->stage_v.reserve(elems));
+  HC_CUDA(c, cudaMemcpyAsync(c->stage_k.ptr, k_host, elems * sizeof(__nv_bfloat16), cudaMemcpyHostToDevice, st));
+  HC_CUDA(c, cudaMemcpyAsync(c->stage_v.ptr, v_host, elems * sizeof(__nv_bfloat16), cudaMemcpyHostToDevice, st));
+  return headcast_append(c, c->stage_k.ptr, c->stage_v.ptr, stream);
+}
+
+int headcast_attend_host(headcast_ctx* c, const void* q_host, void* out_host, void* stream) {
+  if (!c || !q_host || !out_host) return HC_ERR_INVALID_ARG;
+  if (c->state != STATE_SPLIT) return fail(c, HC_ERR_STATE, "head-specific attention needs the split cache");
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int rc = init_host_path(c);
+  if (rc != HC_OK) return rc;
+  const size_t elems = static_cast<size_t>(c->L) * c->H * c->D;
+  HC_CUDA(c, c->stage_q.reserve(elems));
+  HC_CUDA(c, c->stage_out.reserve(elems));
+  const int key = n_filled(c) * 4 + c->sd_valid;
+  for (int g = 0; g < 3; ++g)
+    if (c->sched_group[g].key_filled != key) build_headcast_schedule(c, c->sched_group[g], g);
+  // The heads of one archetype group are copied in (strided: the rows of [L][H][d] hold all heads), attended and copied
+  // out as a unit, so that the next group's queries arrive and the previous group's outputs leave while this group
+  // computes.  Global heads go first: most arithmetic per byte moved.
+  const size_t pitch = static_cast<size_t>(c->H) * c->D * sizeof(__nv_bfloat16);
+  auto copy_group = [&](int g, bool in) -> int {
+    for (int h0 = 0; h0 < c->H;) {
+      auto group_of = [&](int h) { return c->cls[h] == CLS_GLOBAL ? 0 : c->cls[h] == CLS_SPATIAL ? 1 : 2; };
+      if (group_of(h0) != g) {
+        ++h0;
+        continue;
+      }
+      int h1 = h0 + 1;
+      while (h1 < c->H && group_of(h1) == g) ++h1;
+      const size_t off = static_cast<size_t>(h0) * c->D, width = static_cast<size_t>(h1 - h0) * c->D * sizeof(__nv_bfloat16);
+      if (in)
+        HC_CUDA(c, cudaMemcpy2DAsync(c->stage_q.ptr + off, pitch, static_cast<const __nv_bfloat16*>(q_host) + off, pitch, width,
+                                     c->L, cudaMemcpyHostToDevice, c->copy_in));
+      else
+        HC_CUDA(c, cudaMemcpy2DAsync(static_cast<__nv_bfloat16*>(out_host) + off, pitch, c->stage_out.ptr + off, pitch, width,
+                                     c->L, cudaMemcpyDeviceToHost, c->copy_out));
+      h0 = h1;
+    }
+    return HC_OK;
+  };
+  // everything enqueued on `stream` before this call (an append, the previous call's copies) comes first
+  HC_CUDA(c, cudaEventRecord(c->ev_host[0], st));
+  HC_CUDA(c, cudaStreamWaitEvent(c->copy_in, c->ev_host[0], 0));
+  HC_CUDA(c, cudaStreamWaitEvent(c->copy_out, c->ev_host[0], 0));
+  for (int g = 0; g < 3; ++g) {
+    if (c->sched_group[g].items.empty()) continue;
+    if ((rc = copy_group(g, true)) != HC_OK) return rc;
+    HC_CUDA(c, cudaEventRecord(c->ev_host[1 + g], c->copy_in));
+    HC_CUDA(c, cudaStreamWaitEvent(st, c->ev_host[1 + g], 0));
+    if ((rc = run_schedule(c, c->sched_group[g], c->stage_q.ptr, c->stage_out.ptr, false, st)) != HC_OK) return rc;
+    HC_CUDA(c, cudaEventRecord(c->ev_host[4 + g], st));
+    HC_CUDA(c, cudaStreamWaitEvent(c->copy_out, c->ev_host[4 + g], 0));
+    if ((rc = copy_group(g, false)) != HC_OK) return rc;
+  }
+  HC_CUDA(c, cudaEventRecord(c->ev_host[7], c->copy_out));
+  HC_CUDA(c, cudaStreamWaitEvent(st, c->ev_host[7], 0));
+  return HC_OK;
 }
 
 int headcast_export_cache(headcast_ctx* c, int32_t head, void* k_out, void* v_out, int32_t* n_tokens_host, void* stream) {

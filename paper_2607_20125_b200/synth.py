@@ -80,6 +80,33 @@ def wan(resolution: str, seed: int = BASE_SEED, layer: int = 0) -> Workload:
                     labels=_mix(12, (2, 3, 4, 3), seed + 7919 * layer), seed=seed + 7919 * layer)
 
 
+# Head counts out of 30 layers x 12 heads that the paper reports for LongLive at t = 1000 (appendix table of the
+# archetype distribution), rounded so that each row sums to 360: (Sink, Dummy, Spatial, Global).
+REPORTED_HEAD_COUNTS = {"480p": (2, 94, 168, 96), "720p": (2, 98, 167, 93), "1080p": (2, 92, 203, 63)}
+
+
+def reported_mixes(resolution: str, n_layers: int = 30, seed: int = BASE_SEED):
+    """Per-layer label tuples whose totals follow REPORTED_HEAD_COUNTS: the 360 labels are shuffled (seeded) over
+    the layers, so layers differ in their mix and some have no Sink or no Dummy head at all."""
+    counts = REPORTED_HEAD_COUNTS[resolution.lower()]
+    labels = np.repeat(np.arange(4), counts)
+    rng = np.random.Generator(np.random.PCG64([seed, 0x7AB1E6]))
+    labels = rng.permutation(labels).reshape(30, 12)
+    return [tuple(int(v) for v in labels[l % 30]) for l in range(n_layers)]
+
+
+def ablation_labels(labels: Sequence[int]):
+    """The label sets of the paper's archetype ablation: all heads Global; only the Spatial heads sparse; only the
+    Sink and Dummy heads sparse; everything."""
+    lab = np.asarray(labels)
+    return {
+        "all_global": tuple(int(GLOBAL) for _ in lab),
+        "spatial_only": tuple(int(v) if v == SPATIAL else int(GLOBAL) for v in lab),
+        "sink_dummy_only": tuple(int(v) if v in (SINK, DUMMY) else int(GLOBAL) for v in lab),
+        "full": tuple(int(v) for v in lab),
+    }
+
+
 def small(seed: int = BASE_SEED, **kw) -> Workload:
     """A mid-size case for CPU-speed parity runs: ragged tiles, several cells, d=128."""
     base = Workload("small", 6, 128, 13, 22, 4, cell_h=5, cell_w=7,

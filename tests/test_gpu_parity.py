@@ -365,3 +365,43 @@ def test_refresh_of_the_current_block_in_one_block_mode():
         p.append()
     p.check_cache()
     p.check_attention(dense=True)
+
+
+@pytest.mark.parametrize("labels", [None, [orc.GLOBAL] * 6, [orc.SINK, orc.DUMMY, orc.SPATIAL] * 2])
+def test_host_buffer_calls_match_the_oracle(labels):
+    """headcast_append_host / headcast_attend_host: host tensors in, host tensor out, group-wise overlap of the
+    copies with the kernels; cache content stays bit-exact and the outputs meet the same bars as headcast_attend.
+    Pinned and pageable host memory are both accepted."""
+    import torch
+    w = synth.small()
+    lab = w.labels if labels is None else labels
+    p = Pair(w)
+    p.append(2)
+    p.hc.set_labels(lab)
+    p.hc.split_cache()
+    p.cache.split(lab)
+    for i in range(4):  # grows to the full window and rolls once
+        k, v = synth.make_kv(w, p.next_block)
+        host = lambda bits: torch.from_numpy(bits.view(np.int16).copy()).view(torch.bfloat16)
+        kh, vh = host(k), host(v)
+        if i % 2 == 0:
+            kh, vh = kh.pin_memory(), vh.pin_memory()
+        p.hc.append_host(kh, vh)
+        p.cache.append(k, v)
+        p.next_block += 1
+        p.check_cache()
+        q = synth.make_q(w, p.next_block - 1, i)
+        qh = host(q)
+        oh = torch.full(qh.shape, float("nan"), dtype=torch.bfloat16)
+        if i % 2 == 0:
+            qh, oh = qh.pin_memory(), oh.pin_memory()
+        p.hc.attend_host(qh, oh)
+        torch.cuda.current_stream().synchronize()
+        p.hc.check()
+        got = oh.float().numpy().astype(np.float64)
+        assert np.isfinite(got).all(), "columns of some head were not copied back"
+        want = orc.attend(q, p.cache, p.geom)
+        err = np.abs(got - want)
+        assert err.max() <= MAX_ABS and err.mean(axis=(0, 2)).max() <= MEAN_ABS
+        # and the device entry point still agrees afterwards (the two paths share the partial-result buffers)
+        p.check_attention(dense=False, step=i)
