@@ -407,7 +407,7 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const AttnParams 
         const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
         // pass 2: p = 2^(s * c - m), bf16 pack over the first 32 columns of this thread's logits, row sum in fp32
         const uint64_t c2 = pack_f32x2(p.scale_log2e, p.scale_log2e), m2 = pack_f32x2(-m_use, -m_use);
-        uint64_t sum2[2] = {0ull, 0ull};
+        float sum4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
         for (int ch = 0; ch < 2; ++ch) {
           const uint32_t visible = PROXY ? visible_keys<PROXY>(n_valid - ch * 32, tok0 + ch * 32, qy, qx, p.radius, p.grid_w) : 0u;
@@ -439,14 +439,11 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const AttnParams 
             pk[i] = pack_bf16x2(e0, e1);
             // the row sum adds the ROUNDED values: out = sum(p v) / sum(p) is then an exact convex combination of
             // the values even when the reference lags behind the row maximum and the largest p is not exactly 1
-            sum2[i & 1] = add_f32x2(sum2[i & 1], pack_f32x2(__uint_as_float(pk[i] << 16), __uint_as_float(pk[i] & 0xffff0000u)));
+            add_bf16x2_to_f32(pk[i], sum4[(i & 1) * 2], sum4[(i & 1) * 2 + 1]);
           }
           tmem_st16(p_addr + ch * 16, pk);
         }
-        float t0, t1, t2, t3;
-        unpack_f32x2(sum2[0], t0, t1);
-        unpack_f32x2(sum2[1], t2, t3);
-        const float tile_sum = (t0 + t1) + (t2 + t3);
+        const float tile_sum = (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
         l_sum += tile_sum;
         if (PROXY && seg >= p.mid_seg_lo && seg < p.mid_seg_hi && !(seg >= p.last_seg_lo && seg < p.last_seg_hi))
           l_mid += tile_sum;

@@ -290,6 +290,12 @@ __device__ __forceinline__ float ex2_approx(float x) {
   return y;
 }
 // two floats -> packed bf16x2 (lo in bits 0..15), round to nearest even
+// acc_lo += low bf16 of pk, acc_hi += high bf16 of pk, in fp32 (mixed-precision add: no unpacking instructions)
+__device__ __forceinline__ void add_bf16x2_to_f32(uint32_t pk, float& acc_lo, float& acc_hi) {
+  asm("{\n\t.reg .b16 lo, hi;\n\tmov.b32 {lo, hi}, %2;\n\tadd.rn.f32.bf16 %0, lo, %0;\n\tadd.rn.f32.bf16 %1, hi, %1;\n\t}"
+      : "+f"(acc_lo), "+f"(acc_hi)
+      : "r"(pk));
+}
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   uint32_t r;
   asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
