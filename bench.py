@@ -99,6 +99,15 @@ class ClockSampler:
                 "samples": len(self.samples)}
 
 
+def max_over_ranks(value: float, dist, torch, device) -> float:
+    """The slowest rank's value (every rank gets it); the identity on a single process."""
+    if dist is None:
+        return float(value)
+    t = torch.tensor([value], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
 def to_dev(bits, torch):
     return torch.from_numpy(bits.view(np.int16)).view(torch.bfloat16).cuda()
 
@@ -413,11 +422,7 @@ def main():
         dist.barrier()
     hc.check()
     launches = hc.launch_count() - launches0
-    total_ms = float(np.sum(step_ms))
-    if dist is not None:
-        tt = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        total_ms = float(tt.item())
+    total_ms = max_over_ranks(float(np.sum(step_ms)), dist, torch, "cuda")
     ms_per_step = total_ms / args.steps
     attend_ms = float(np.mean([s - (append_ms[i // STEPS_PER_BLOCK] if i % STEPS_PER_BLOCK == 0 else 0.0)
                                for i, s in enumerate(step_ms)]))
@@ -472,11 +477,7 @@ def main():
         if i >= 0:
             e2e_ms.append(a.elapsed_time(b))
     hc.check()
-    e2e = float(np.sum(e2e_ms)) / e2e_steps
-    if dist is not None:
-        tt = torch.tensor([e2e], device="cuda", dtype=torch.float64)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        e2e = float(tt.item())
+    e2e = max_over_ranks(float(np.sum(e2e_ms)) / e2e_steps, dist, torch, "cuda")
     q_bytes = L * H * D * 2
 
     if rank != 0:

@@ -1,0 +1,69 @@
+"""The multi-process side of bench.py, on CPU: the path does not shard, `--gpus N` runs N independent replicas and
+only the timing is reduced (maximum over ranks).  Two gloo ranks check that reduction, and two processes launched
+the way the driver launches the reference arm check that rank 0 alone prints the JSON line."""
+import json
+import os
+import subprocess
+import sys
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+RANK_SCRIPT = r"""
+import os, sys
+sys.path.insert(0, os.environ["HC_ROOT"])
+import torch
+import torch.distributed as dist
+import bench
+dist.init_process_group("gloo", init_method="tcp://127.0.0.1:" + os.environ["HC_PORT"],
+                        rank=int(os.environ["RANK"]), world_size=int(os.environ["WORLD_SIZE"]))
+rank = dist.get_rank()
+mine = [3.5, 7.25][rank]
+got = bench.max_over_ranks(mine, dist, torch, "cpu")
+assert got == 7.25, (rank, got)
+assert bench.max_over_ranks(mine, None, torch, "cpu") == mine
+dist.barrier()
+dist.destroy_process_group()
+print("rank", rank, "ok")
+"""
+
+
+def _free_port() -> int:
+    import socket
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def _spawn(code_or_args, rank, world, port, code=True):
+    env = dict(os.environ, RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE=str(world), MASTER_ADDR="127.0.0.1",
+               MASTER_PORT=str(port), HC_PORT=str(port), HC_ROOT=ROOT)
+    args = [sys.executable, "-c", code_or_args] if code else [sys.executable] + code_or_args
+    return subprocess.Popen(args, cwd=ROOT, env=env, stdout=subprocess.PIPE, stderr=subprocess.PIPE, text=True)
+
+
+def test_timing_is_the_maximum_over_two_gloo_ranks():
+    port = _free_port()
+    procs = [_spawn(RANK_SCRIPT, r, 2, port) for r in range(2)]
+    outs = [p.communicate(timeout=240) for p in procs]
+    for r, (p, (out, err)) in enumerate(zip(procs, outs)):
+        assert p.returncode == 0, err[-2000:]
+        assert f"rank {r} ok" in out
+
+
+def test_reference_arm_prints_one_line_from_rank_zero_only():
+    port = _free_port()
+    args = [os.path.join(ROOT, "bench.py"), "--impl", "reference", "--workload", "tiny", "--gpus", "2", "--steps", "1",
+            "--warmup", "3"]
+    procs = [_spawn(args, r, 2, port, code=False) for r in range(2)]
+    outs = [p.communicate(timeout=600) for p in procs]
+    for p, (out, err) in zip(procs, outs):
+        assert p.returncode == 0, err[-2000:]
+    assert outs[1][0].strip() == "", "ranks other than 0 exit without work or output"
+    lines = [l for l in outs[0][0].splitlines() if l.strip()]
+    assert len(lines) == 1
+    line = json.loads(lines[0])
+    assert line["impl"] == "reference" and line["n_gpus"] == 2 and line["unit"] == "ms"
+    assert line["higher_is_better"] is False and line["value"] > 0
+    assert line["cpu_baseline"]["kind"] == "oracle" and line["cpu_baseline"]["value"] == line["value"]
+    assert line["e2e"] == {"value": line["value"], "unit": "ms", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}
+    assert line["config"]["workload"] == "tiny"
