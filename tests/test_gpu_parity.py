@@ -405,3 +405,34 @@ def test_host_buffer_calls_match_the_oracle(labels):
         assert err.max() <= MAX_ABS and err.mean(axis=(0, 2)).max() <= MEAN_ABS
         # and the device entry point still agrees afterwards (the two paths share the partial-result buffers)
         p.check_attention(dense=False, step=i)
+
+
+@pytest.mark.parametrize("case", range(12))
+def test_seeded_random_shapes(case):
+    """Shapes nobody picked by hand: grid, cell size, head count and head_dim, window, frames per block, label mix
+    (classes may be missing), fill level at the split, number of rolls and the Sink/Dummy mode are drawn from a
+    seeded generator; every stage of the pipeline must still match the oracle."""
+    rng = np.random.default_rng(4200 + case)
+    n_heads = int(rng.integers(2, 7))
+    w = synth.Workload(
+        name=f"random{case}", n_heads=n_heads, head_dim=int(rng.choice([64, 128])),
+        grid_h=int(rng.integers(3, 15)), grid_w=int(rng.integers(4, 21)), n_blocks=int(rng.integers(2, 6)),
+        frames_per_block=int(rng.integers(1, 4)), cell_h=int(rng.integers(2, 8)), cell_w=int(rng.integers(2, 8)),
+        labels=tuple(int(v) for v in rng.integers(0, 4, size=n_heads)), sink_alpha=8.0, seed=synth.BASE_SEED + case)
+    fill = int(rng.integers(1, w.n_blocks + 1))
+    extra = int(rng.integers(1, 2 * w.n_blocks))
+    run_pipeline(w, fill=fill, extra=extra, sd_mode=int(rng.integers(0, 2)))
+    # classification of the same shape (needs two cached blocks): scores within the bars; labels must agree wherever
+    # the float64 decision is not within the score tolerance of a threshold
+    cfill = max(2, fill)
+    p = Pair(w)
+    p.append(cfill)
+    q = synth.make_q(w, cfill - 1, 0)
+    labels, scores = p.hc.classify(to_dev(q))
+    want_labels, want = orc.classify(q, p.cache, p.geom)
+    d = np.abs(scores.astype(np.float64) - want)
+    assert d[:, [0, 1, 2, 6, 7, 8, 9]].max() <= 5e-3, d
+    assert d[:, [3, 5]].max() <= 1e-2 and d[:, 4].max() <= 2e-3, d
+    theta = np.array([0.95, 0.95, 0.95])
+    decisive = (np.abs(want[:, :3] - theta).min(axis=1) > 1e-2) & (np.abs(want[:, 3] - 0.755) > 2e-2)
+    assert all(int(a) == int(b) for a, b, ok in zip(labels, want_labels, decisive) if ok), (labels, want_labels)
