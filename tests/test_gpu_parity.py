@@ -434,5 +434,5 @@ def test_seeded_random_shapes(case):
     assert d[:, [0, 1, 2, 6, 7, 8, 9]].max() <= 5e-3, d
     assert d[:, [3, 5]].max() <= 1e-2 and d[:, 4].max() <= 2e-3, d
     theta = np.array([0.95, 0.95, 0.95])
-    decisive = (np.abs(want[:, :3] - theta).min(axis=1) > 1e-2) & (np.abs(want[:, 3] - 0.755) > 2e-2)
+    decisive = (np.abs(want[:, :3] - theta).min(axis=1) > 1e-2) & (np.abs(want[:, 5] - 0.755) > 2e-2)
     assert all(int(a) == int(b) for a, b, ok in zip(labels, want_labels, decisive) if ok), (labels, want_labels)
