@@ -564,4 +564,72 @@ combine_kernel(const CombineEntry* entries, const CellGeom* cells, const float* 
   *reinterpret_cast<uint4*>(out + (static_cast<size_t>(token) * n_heads + e.head) * D + c * 8) = o4;
 }
 
+// Classification: the reference attention (Eq. 2) and the Sink / Dummy proxies from ONE sweep over the keys.  The
+// sweep is cut into key ranges tagged first block / middle blocks / newest block, every range leaves an unnormalised
+// partial result, and this kernel merges them three ways per query row:
+//   all ranges -> reference output, pass 0;  first block only -> Sink proxy, pass 1;  newest block only -> Dummy
+//   proxy, pass 2;  each with its log-sum-exp (natural log).
+// parts[first_part .. first_part + n_parts) of a group list (partial slot, tag); a group is one 256-row query pair.
+struct ClsPart {
+  int32_t slot, tag;  // tag: 0 first block, 1 middle, 2 newest block
+};
+struct ClsGroup {
+  int32_t head, q_start, q_count[2], first_part, n_parts;
+};
+
+template <int D>
+__global__ void __launch_bounds__(COMBINE_ROWS * (D / 8))
+cls_combine_kernel(const ClsGroup* groups, const ClsPart* parts, const float* part_o, const float2* part_ml, float* f32_o,
+                   float* f32_lse, int n_heads, int block_tokens) {
+  constexpr int CHUNKS = D / 8;
+  constexpr int BLOCKS_PER_TILE = 128 / COMBINE_ROWS;
+  const ClsGroup g = groups[blockIdx.x / (2 * BLOCKS_PER_TILE)];
+  const int sub = (blockIdx.x / BLOCKS_PER_TILE) & 1;
+  const int r = (blockIdx.x % BLOCKS_PER_TILE) * COMBINE_ROWS + threadIdx.x / CHUNKS;
+  const int c = threadIdx.x % CHUNKS;
+  if (r >= g.q_count[sub]) return;
+  const ClsPart* pp = parts + g.first_part;
+  float m[3] = {-INFINITY, -INFINITY, -INFINITY};  // all, first, newest
+  for (int i = 0; i < g.n_parts; ++i) {
+    const float mi = part_ml[static_cast<size_t>(pp[i].slot) * 256 + sub * 128 + r].x;
+    m[0] = fmaxf(m[0], mi);
+    if (pp[i].tag == 0) m[1] = fmaxf(m[1], mi);
+    if (pp[i].tag == 2) m[2] = fmaxf(m[2], mi);
+  }
+  float acc[3][8], l[3] = {0.f, 0.f, 0.f};
+#pragma unroll
+  for (int k = 0; k < 3; ++k)
+#pragma unroll
+    for (int j = 0; j < 8; ++j) acc[k][j] = 0.f;
+  for (int i = 0; i < g.n_parts; ++i) {
+    const size_t row = static_cast<size_t>(pp[i].slot) * 256 + sub * 128 + r;
+    const float2 ml = part_ml[row];
+    if (ml.x == -INFINITY) continue;
+    const float4* src = reinterpret_cast<const float4*>(part_o + row * D + c * 8);
+    const float4 a = src[0], b = src[1];
+    const float v[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+#pragma unroll
+    for (int k = 0; k < 3; ++k) {
+      const bool in_set = (k == 0) || (k == 1 && pp[i].tag == 0) || (k == 2 && pp[i].tag == 2);
+      if (!in_set) continue;
+      const float wgt = ex2_approx(ml.x - m[k]);
+      l[k] += wgt * ml.y;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) acc[k][j] += wgt * v[j];
+    }
+  }
+  const int token = g.q_start + sub * 128 + r;
+  const size_t lh = static_cast<size_t>(block_tokens) * n_heads;
+  const size_t idx = static_cast<size_t>(token) * n_heads + g.head;
+  const float ln2 = 0.6931471805599453f;
+#pragma unroll
+  for (int k = 0; k < 3; ++k) {
+    const float inv = l[k] > 0.f ? 1.f / l[k] : 0.f;
+    float4* dst = reinterpret_cast<float4*>(f32_o + (k * lh + idx) * D + c * 8);
+    dst[0] = make_float4(acc[k][0] * inv, acc[k][1] * inv, acc[k][2] * inv, acc[k][3] * inv);
+    dst[1] = make_float4(acc[k][4] * inv, acc[k][5] * inv, acc[k][6] * inv, acc[k][7] * inv);
+    if (c == 0) f32_lse[k * lh + idx] = (l[k] > 0.f) ? m[k] * ln2 + __logf(l[k]) : -INFINITY;
+  }
+}
+
 }  // namespace hc

@@ -50,9 +50,13 @@ struct Schedule {
   std::vector<WorkItem> items;
   std::vector<int32_t> cta_first;
   std::vector<CombineEntry> combine;
+  std::vector<ClsGroup> cls_groups;  // classification only: key ranges of one query pair, merged three ways
+  std::vector<ClsPart> cls_parts;
   DevBuf<WorkItem> items_dev;
   DevBuf<int32_t> cta_first_dev;
   DevBuf<CombineEntry> combine_dev;
+  DevBuf<ClsGroup> cls_groups_dev;
+  DevBuf<ClsPart> cls_parts_dev;
   int n_slots = 0;
   bool uploaded = false;
   double flops = 0.0;
@@ -60,6 +64,8 @@ struct Schedule {
     items_dev.release();
     cta_first_dev.release();
     combine_dev.release();
+    cls_groups_dev.release();
+    cls_parts_dev.release();
   }
 };
 
@@ -190,6 +196,8 @@ int build_maps(headcast_ctx* c) {
 struct Proto {  // one (head, query-tile pair, key range) before it is cut into parts
   WorkItem w;
   int n_tiles;
+  int cls_group = -1;  // classification: every piece writes a partial result that belongs to this group ...
+  int cls_tag = 0;     // ... with this tag (0 first block, 1 middle blocks, 2 newest block)
 };
 
 void add_query_pairs(std::vector<Proto>& out, WorkItem base, int n_queries, int n_tiles) {
@@ -261,9 +269,12 @@ void finalize_schedule(headcast_ctx* c, Schedule& s, std::vector<Proto>& protos,
       base_total += item_cost(p.w);
       largest = std::max(largest, item_cost(p.w));
     }
+    struct RawPart { int group, slot, tag; };
+    std::vector<RawPart> cls_raw;
     auto lay_out = [&](double quota) -> double {
       for (auto& bin : bins) bin.clear();
       s.combine.clear();
+      cls_raw.clear();
       s.n_slots = 0;
       int cta = 0;
       double room = quota, last_load = 0.0;
@@ -294,11 +305,20 @@ void finalize_schedule(headcast_ctx* c, Schedule& s, std::vector<Proto>& protos,
           w.tile_begin = begin;
           w.tile_end = begin + take;
           parts.push_back(std::make_pair(cta, w));
-          const bool cut = (take < left) || begin > 0;
+          const bool cut = (take < left) || begin > 0 || p.cls_group >= 0;
           const double cost = per_tile * take + overhead + (cut ? PARTIAL_EXTRA : 0.0);
           room -= cost;
           if (cta == n_cta - 1) last_load += cost;
           begin += take;
+        }
+        if (p.cls_group >= 0) {
+          for (auto& pr : parts) {
+            pr.second.out_mode = OUT_PARTIAL;
+            pr.second.out_slot = s.n_slots++;
+            bins[pr.first].push_back(pr.second);
+            cls_raw.push_back({p.cls_group, pr.second.out_slot, p.cls_tag});
+          }
+          continue;
         }
         if (parts.size() == 1) {
           bins[parts[0].first].push_back(parts[0].second);
@@ -332,6 +352,16 @@ void finalize_schedule(headcast_ctx* c, Schedule& s, std::vector<Proto>& protos,
       if (lay_out(mid) <= mid) hi = mid; else lo = mid;
     }
     lay_out(hi);
+    // classification: the pieces of every group, in group order
+    std::stable_sort(cls_raw.begin(), cls_raw.end(), [](const RawPart& a, const RawPart& b) { return a.group < b.group; });
+    s.cls_parts.clear();
+    for (ClsGroup& g : s.cls_groups) g.n_parts = 0;
+    for (const RawPart& rp : cls_raw) {
+      ClsGroup& g = s.cls_groups[rp.group];
+      if (g.n_parts == 0) g.first_part = static_cast<int32_t>(s.cls_parts.size());
+      ++g.n_parts;
+      s.cls_parts.push_back(ClsPart{rp.slot, rp.tag});
+    }
   } else {
     typedef std::pair<double, int> Load;
     std::priority_queue<Load, std::vector<Load>, std::greater<Load>> pq;
@@ -417,6 +447,14 @@ int upload_schedule(headcast_ctx* c, Schedule& s, cudaStream_t st) {
   if (!s.combine.empty())
     HC_CUDA(c, cudaMemcpyAsync(s.combine_dev.ptr, s.combine.data(), s.combine.size() * sizeof(CombineEntry),
                                cudaMemcpyHostToDevice, st));
+  if (!s.cls_groups.empty()) {
+    HC_CUDA(c, s.cls_groups_dev.reserve(s.cls_groups.size()));
+    HC_CUDA(c, s.cls_parts_dev.reserve(std::max<size_t>(1, s.cls_parts.size())));
+    HC_CUDA(c, cudaMemcpyAsync(s.cls_groups_dev.ptr, s.cls_groups.data(), s.cls_groups.size() * sizeof(ClsGroup),
+                               cudaMemcpyHostToDevice, st));
+    HC_CUDA(c, cudaMemcpyAsync(s.cls_parts_dev.ptr, s.cls_parts.data(), s.cls_parts.size() * sizeof(ClsPart),
+                               cudaMemcpyHostToDevice, st));
+  }
   if (s.n_slots > 0) {
     HC_CUDA(c, c->part_o.reserve(static_cast<size_t>(s.n_slots) * 256 * c->D));
     HC_CUDA(c, c->part_ml.reserve(static_cast<size_t>(s.n_slots) * 256));
@@ -489,6 +527,17 @@ int run_schedule(headcast_ctx* c, Schedule& s, const void* q, void* out, bool pr
   else
     rc = proxy ? launch_attn_t<64, true>(c, p, st) : launch_attn_t<64, false>(c, p, st);
   if (rc != HC_OK) return rc;
+  if (!s.cls_groups.empty()) {
+    const unsigned blocks = static_cast<unsigned>(s.cls_groups.size()) * 2 * (128 / COMBINE_ROWS);
+    if (c->D == 128)
+      cls_combine_kernel<128><<<blocks, COMBINE_ROWS * 16, 0, st>>>(s.cls_groups_dev.ptr, s.cls_parts_dev.ptr, c->part_o.ptr,
+                                                                    c->part_ml.ptr, c->cls_o.ptr, c->cls_lse.ptr, c->H, c->L);
+    else
+      cls_combine_kernel<64><<<blocks, COMBINE_ROWS * 8, 0, st>>>(s.cls_groups_dev.ptr, s.cls_parts_dev.ptr, c->part_o.ptr,
+                                                                  c->part_ml.ptr, c->cls_o.ptr, c->cls_lse.ptr, c->H, c->L);
+    HC_CUDA(c, cudaGetLastError());
+    ++c->launches;
+  }
   if (!s.combine.empty()) {
     const unsigned blocks = static_cast<unsigned>(s.combine.size()) * (128 / COMBINE_ROWS);
     if (c->D == 128)
@@ -855,25 +904,56 @@ int headcast_classify(headcast_ctx* c, const void* q, int32_t* labels_host, floa
   HC_CUDA(c, c->cls_scores.reserve(static_cast<size_t>(c->H) * HC_N_SCORES));
   HC_CUDA(c, c->cls_labels.reserve(c->H));
   const int newest = c->slots.back();
-  {  // reference (Eq. 2), Sink proxy and Dummy proxy share one launch
+  const int cls_key = n_filled(c) * 64 + newest;  // the work lists depend on the fill and on where the newest block sits
+  if (c->sched_cls.key_filled != cls_key) {
+    // Reference (Eq. 2), Sink proxy and Dummy proxy from one sweep over the keys: the sweep is cut into the first
+    // block, the middle blocks and the newest block (physical ring slots: the middle ones are one or two runs),
+    // every piece leaves a partial result and cls_combine_kernel merges them three ways.
     std::vector<Proto> protos;
-    for (int h = 0; h < c->H; ++h) {
-      WorkItem w = range_item(h, MAP_MONO, h * c->D, 0, n_filled(c) * c->L);
-      w.out_mode = OUT_F32_LSE;
-      w.out_slot = 0;
-      add_query_pairs(protos, w, c->L, w.tiles_per_seg);
-      w = range_item(h, MAP_MONO, h * c->D, 0, c->L);
-      w.out_mode = OUT_F32_LSE;
-      w.out_slot = 1;
-      add_query_pairs(protos, w, c->L, w.tiles_per_seg);
-      w = range_item(h, MAP_MONO, h * c->D, static_cast<long long>(newest) * c->L, c->L);
-      w.out_mode = OUT_F32_LSE;
-      w.out_slot = 2;
-      add_query_pairs(protos, w, c->L, w.tiles_per_seg);
-    }
-    finalize_schedule(c, c->sched_cls, protos, false);
+    Schedule& s = c->sched_cls;
+    s.cls_groups.clear();
+    const int nf = n_filled(c);
+    struct Range { int slot_lo, slot_hi, tag; };
+    std::vector<Range> ranges;
+    ranges.push_back({0, 1, 0});
+    if (newest > 1) ranges.push_back({1, newest, 1});
+    if (newest + 1 < nf) ranges.push_back({newest + 1, nf, 1});
+    if (newest != 0) ranges.push_back({newest, newest + 1, 2});
+    for (int h = 0; h < c->H; ++h)
+      for (int q0 = 0; q0 < c->L; q0 += 256) {
+        ClsGroup g;
+        g.head = h;
+        g.q_start = q0;
+        g.q_count[0] = std::min(128, c->L - q0);
+        g.q_count[1] = std::max(0, std::min(128, c->L - q0 - 128));
+        g.first_part = 0;
+        g.n_parts = 0;
+        const int group = static_cast<int>(s.cls_groups.size());
+        s.cls_groups.push_back(g);
+        for (const Range& r : ranges) {
+          WorkItem w = range_item(h, MAP_MONO, h * c->D, static_cast<long long>(r.slot_lo) * c->L, (r.slot_hi - r.slot_lo) * c->L);
+          Proto p;
+          p.w = w;
+          p.w.q_start[0] = q0;
+          p.w.q_start[1] = q0 + 128;
+          p.w.q_count[0] = g.q_count[0];
+          p.w.q_count[1] = g.q_count[1];
+          p.n_tiles = w.tiles_per_seg;
+          p.w.tile_begin = 0;
+          p.w.tile_end = p.n_tiles;
+          p.cls_group = group;
+          p.cls_tag = r.tag;
+          protos.push_back(p);
+        }
+      }
+    finalize_schedule(c, s, protos, true);
+    s.key_filled = cls_key;
   }
-  {  // Spatial proxy: per query-tile pair, the band of grid rows within r of any of its queries, in every cached frame
+  // the reference sweep is on its way before the host builds the proxy's work list
+  int rc = run_schedule(c, c->sched_cls, q, nullptr, false, st);
+  if (rc != HC_OK) return rc;
+  if (c->sched_proxy.key_filled != cls_key) {
+    // Spatial proxy: per query-tile pair, the band of grid rows within r of any of its queries, in every cached frame
     std::vector<Proto> protos;
     const int r = c->cfg.proxy_radius;
     for (int h = 0; h < c->H; ++h)
@@ -901,9 +981,8 @@ int headcast_classify(headcast_ctx* c, const void* q, int32_t* labels_host, floa
         protos.push_back(p);
       }
     finalize_schedule(c, c->sched_proxy, protos, false);
+    c->sched_proxy.key_filled = cls_key;
   }
-  int rc = run_schedule(c, c->sched_cls, q, nullptr, false, st);
-  if (rc != HC_OK) return rc;
   rc = run_schedule(c, c->sched_proxy, q, nullptr, true, st);
   if (rc != HC_OK) return rc;
   {
