@@ -345,13 +345,40 @@ void finalize_schedule(headcast_ctx* c, Schedule& s, std::vector<Proto>& protos,
       }
       return last_load;
     };
-    double lo = base_total / n_cta, hi = base_total / n_cta + largest + ITEM_OVERHEAD + PARTIAL_EXTRA;
-    while (lay_out(hi) > hi) hi *= 1.25;
+    // The share is found by bisection between the ideal share and one that surely fits.  "Fits" is not quite monotone
+    // in the share (room an item could not be cut into is lost, and how much depends on where the cuts fall), so the
+    // bisection can settle on a share far too large and leave many CTAs idle; when that happens the shares are
+    // scanned upwards from the ideal one instead, coarsely and then finely, and the first that fits is taken.
+    const double ideal = base_total / n_cta;
+    auto fits = [&](double share) { return lay_out(share) <= share; };
+    auto idle_ctas = [&]() {
+      int n = 0;
+      for (const auto& bin : bins) n += bin.empty();
+      return n;
+    };
+    double lo = ideal, hi = ideal + largest + ITEM_OVERHEAD + PARTIAL_EXTRA;
+    while (!fits(hi)) hi *= 1.25;
     for (int iter = 0; iter < 24 && hi - lo > 0.25; ++iter) {
       const double mid = 0.5 * (lo + hi);
-      if (lay_out(mid) <= mid) hi = mid; else lo = mid;
+      if (fits(mid)) hi = mid; else lo = mid;
     }
     lay_out(hi);
+    if (idle_ctas() > std::max(2, n_cta / 20)) {
+      double share = ideal;
+      int step = 0;
+      while (!fits(share) && step < 400) share = ideal * (1.0 + 0.02 * ++step);
+      if (step > 0) {
+        const double below = ideal * (1.0 + 0.02 * (step - 1));
+        for (int k = 1; k < 8; ++k) {
+          const double fine = below + (share - below) * k / 8.0;
+          if (fits(fine)) {
+            share = fine;
+            break;
+          }
+        }
+      }
+      lay_out(share);
+    }
     // classification: the pieces of every group, in group order
     std::stable_sort(cls_raw.begin(), cls_raw.end(), [](const RawPart& a, const RawPart& b) { return a.group < b.group; });
     s.cls_parts.clear();
