@@ -411,7 +411,7 @@ void finalize_schedule(headcast_ctx* c, Schedule& s, std::vector<Proto>& protos,
       double all_cost = 0.0;
       for (const Proto& p : protos) {
         all_cost += item_cost(p.w);
-        if (p.w.cell >= 0 || p.cls_group >= 0) continue;
+        if (p.w.cell >= 0) continue;
         auto it = std::find_if(streams.begin(), streams.end(), [&](const Stream& st) { return st.map == p.w.kv_map && st.head == p.w.head; });
         if (it == streams.end()) {
           const long long segs = (p.n_tiles + p.w.tiles_per_seg - 1) / p.w.tiles_per_seg;
@@ -443,7 +443,7 @@ void finalize_schedule(headcast_ctx* c, Schedule& s, std::vector<Proto>& protos,
         for (size_t ph = 0; ph < phase_cost.size(); ++ph) {
           if (phase_cost[ph] < 60.0 * n_cta) continue;
           auto in_phase = [&](const Proto& p) {
-            if (p.w.cell >= 0 || p.cls_group >= 0) return false;
+            if (p.w.cell >= 0) return false;
             for (const Stream& st : streams)
               if (st.map == p.w.kv_map && st.head == p.w.head) return st.phase == static_cast<int>(ph);
             return false;
