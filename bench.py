@@ -465,7 +465,7 @@ def main():
     host_out = torch.empty_like(host_q[0]).pin_memory()
     e2e_steps = min(args.steps, 40)
     e2e_ms = []
-    for i in range(-3, e2e_steps):
+    for i in range(-STEPS_PER_BLOCK, e2e_steps):  # the warm-up includes one append
         flush()
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a.record()
