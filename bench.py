@@ -351,6 +351,10 @@ def main():
         phases["classify_ms"] = a.elapsed_time(b)
         phases["classify_first_call_ms"] = t_first
         phases["labels_match_planted"] = bool(tuple(int(v) for v in labels) == tuple(w.labels))
+        # how far every thresholded quantity of every head is from its threshold (cosines vs 0.95, score vs 0.755)
+        sc = np.asarray(scores, dtype=np.float64)
+        phases["classify_margins"] = {"min_abs_cos_minus_theta": float(np.abs(sc[:, :3] - 0.95).min()),
+                                      "min_abs_score_minus_theta": float(np.abs(sc[:, 5] - 0.755).min())}
         t = timed(torch, lambda: hc.append(*kv[w.n_blocks]), flush, 5)  # monolithic ring append (rolls)
         phases["append_monolithic_ms"] = t
         phases["append_monolithic_gbs"] = 2 * block_bytes / t / 1e6
@@ -384,15 +388,16 @@ def main():
     for _ in range(args.warmup):
         step()
     hc.check()
-    # append throughput without launch gaps: 16 launches back to back inside one event pair (1.3 GB at 480P, > L2)
+    # append throughput without launch gaps: 200 launches back to back inside one event pair (16 GB at 480P, > L2)
+    n_b2b = 200
     flush()
     a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     a.record()
-    for i in range(16):
+    for i in range(n_b2b):
         hc.append(*kv[w.n_blocks + i % n_extra])
     b.record()
     b.synchronize()
-    phases["append_split_back_to_back_ms"] = a.elapsed_time(b) / 16
+    phases["append_split_back_to_back_ms"] = a.elapsed_time(b) / n_b2b
     phases["append_split_back_to_back_gbs"] = append_bytes / phases["append_split_back_to_back_ms"] / 1e6
     state["i"] = 0
     if dist is not None:
@@ -483,6 +488,7 @@ def main():
     if rank != 0:
         return
     achieved = flops / kern / 1e9
+    pct = lambda xs: {"p10": float(np.percentile(xs, 10)), "p50": float(np.percentile(xs, 50)), "p90": float(np.percentile(xs, 90))}
     line = {
         "metric": METRIC, "value": ms_per_step, "unit": "ms", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
@@ -494,6 +500,7 @@ def main():
         "clocks": clocks.summary(),
         "e2e": {"value": e2e, "unit": "ms", "h2d_bytes_per_step": q_bytes + block_bytes // STEPS_PER_BLOCK, "d2h_bytes_per_step": q_bytes},
         "gpu_launches": int(launches),
+        "spread": {"step_ms": pct(step_ms), "attention_kernel_ms": pct(kernel_ms), "e2e_ms": pct(e2e_ms)},
         "roofline": {"bound": "tensor", "kernel": "attn_kernel (tcgen05)", "achieved": achieved, "peak": peaks["tflops"],
                      "unit": "TFLOP/s", "frac": achieved / peaks["tflops"], "peak_source": peaks["source"] + " (burst bf16 GEMM)",
                      "frac_of_sustained": achieved / peaks["tflops_sustained"] if peaks["tflops_sustained"] else None,
