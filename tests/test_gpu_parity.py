@@ -436,3 +436,24 @@ def test_seeded_random_shapes(case):
     theta = np.array([0.95, 0.95, 0.95])
     decisive = (np.abs(want[:, :3] - theta).min(axis=1) > 1e-2) & (np.abs(want[:, 5] - 0.755) > 2e-2)
     assert all(int(a) == int(b) for a, b, ok in zip(labels, want_labels, decisive) if ok), (labels, want_labels)
+
+
+def test_maximum_head_and_block_counts():
+    """The largest context the header allows: 64 heads and a 32-block window (small grid so that the oracle stays
+    quick).  Fills the whole window, splits, rolls past the end of the ring, and classifies."""
+    rng = np.random.default_rng(77)
+    labels = tuple(int(v) for v in rng.integers(0, 4, size=64))
+    w = synth.Workload(name="limits", n_heads=64, head_dim=64, grid_h=5, grid_w=7, n_blocks=32, frames_per_block=2,
+                       cell_h=3, cell_w=4, labels=labels, sink_alpha=8.0, seed=synth.BASE_SEED + 99)
+    rows = np.arange(0, w.block_tokens, 3)
+    p = run_pipeline(w, fill=32, extra=3, rows=rows)
+    assert p.hc.n_filled() == 32
+    q = synth.make_q(w, p.next_block - 1, 1)
+    c = Pair(w)
+    c.append(32)
+    got_labels, scores = c.hc.classify(to_dev(synth.make_q(w, 31, 0)))
+    want_labels, want = orc.classify(synth.make_q(w, 31, 0), c.cache, c.geom)
+    d = np.abs(scores.astype(np.float64) - want)
+    assert d[:, [0, 1, 2, 6, 7, 8, 9]].max() <= 5e-3 and d[:, [3, 5]].max() <= 1e-2 and d[:, 4].max() <= 2e-3
+    decisive = (np.abs(want[:, :3] - 0.95).min(axis=1) > 1e-2) & (np.abs(want[:, 5] - 0.755) > 2e-2)
+    assert all(int(a) == int(b) for a, b, ok in zip(got_labels, want_labels, decisive) if ok)
