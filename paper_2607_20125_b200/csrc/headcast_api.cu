@@ -233,13 +233,17 @@ WorkItem range_item(int head, int map, int x0, long long row0, int n_keys) {
 // Cost model of the scheduler, in units of the time one key tile takes with both query tiles in flight
 // (fitted to per-item timings from headcast_read_trace on B200): a lone query tile still needs 0.82 of that
 // because the chain S -> softmax -> P -> next S is latency bound; every item pays for its query load, pipeline
-// fill and epilogue; a partial result costs an extra round trip through global memory.
+// fill and epilogue; a partial result costs an extra round trip through global memory; the tiles of Spatial items
+// measure 5 % slower and the CTAs that hold nothing else finished last, hence the factor on them.
 constexpr double TILE_COST_PAIR = 1.0, TILE_COST_SINGLE = 0.82;
 constexpr double ITEM_OVERHEAD = 3.5, ITEM_OVERHEAD_SINGLE = 2.5;
 constexpr double PARTIAL_EXTRA = 1.0;
+constexpr double SPATIAL_FACTOR = 1.10;  // tiles of Spatial items (queries gathered by cell, short cell-major key runs) take longer
 constexpr int MIN_PART_TILES = 4;  // never cut a key range into pieces shorter than this
 
-double tile_cost(const WorkItem& w) { return w.q_count[1] > 0 ? TILE_COST_PAIR : TILE_COST_SINGLE; }
+double tile_cost(const WorkItem& w) {
+  return (w.q_count[1] > 0 ? TILE_COST_PAIR : TILE_COST_SINGLE) * (w.cell >= 0 ? SPATIAL_FACTOR : 1.0);
+}
 
 double item_overhead(const WorkItem& w) { return w.q_count[1] > 0 ? ITEM_OVERHEAD : ITEM_OVERHEAD_SINGLE; }
 
