@@ -244,6 +244,39 @@ def run_rollout(args):
     t["headcast_ms"] = a.elapsed_time(b)
     launches = sum(hc.launch_count() for hc in layers) - launches0
     flops = sum(hc.attend_flops(False) for hc in layers)
+    if args.graphs:
+        # The same steady-state blocks replayed from CUDA graphs: one graph per layer and ring position (the slot a new
+        # block lands in cycles with period n_blocks - 1, and after that many appends the host-side ring is back where
+        # it started, so capture leaves the contexts consistent).  Capture records the launches, it does not run them.
+        period = base.n_blocks - 1
+        graphs = []
+        try:
+            for hc in layers:
+                per_layer = []
+                for ph in range(period):
+                    gr = torch.cuda.CUDAGraph()
+                    with torch.cuda.graph(gr):
+                        hc.append(*kv[ph % pool])
+                        for s_ in range(STEPS_PER_BLOCK):
+                            hc.attend(qs[s_], out)
+                    per_layer.append(gr)
+                graphs.append(per_layer)
+            torch.cuda.synchronize()
+            for per_layer in graphs:  # one warm replay of everything
+                per_layer[0].replay()
+            torch.cuda.synchronize()
+            a, b = ev(), ev()
+            a.record()
+            for blk in range(args.blocks):
+                for per_layer in graphs:
+                    per_layer[blk % period].replay()
+            b.record(); b.synchronize()
+            t["headcast_graph_ms"] = a.elapsed_time(b)
+            t["graph_launches"] = args.blocks * len(layers)
+        except Exception as exc:  # report, do not hide
+            t["headcast_graph_ms"] = None
+            t["graph_error"] = str(exc)[:200]
+        graphs = None
     a, b = ev(), ev()
     a.record()
     for blk in range(args.blocks):
@@ -286,6 +319,8 @@ def main():
                     help="rollout: 2/3/4/3 heads per layer, or the 360-head distribution the paper reports for LongLive at 720P")
     ap.add_argument("--ablation", default="full", choices=["full", "all_global", "spatial_only", "sink_dummy_only"],
                     help="rollout: which archetypes stay sparse (the paper's archetype ablation); the rest become Global")
+    ap.add_argument("--graphs", action="store_true",
+                    help="rollout: also replay the steady-state blocks from CUDA graphs (one per layer and ring position)")
     ap.add_argument("--ablations", action="store_true",
                     help="single layer: also time headcast_attend for the label sets of the paper's archetype ablation")
     ap.add_argument("--no-cpu-baseline", action="store_true")
