@@ -65,6 +65,7 @@ struct AttnParams {
   __nv_bfloat16* out;      // [L][H][d]
   float* part_o;           // [slot][256][d] unnormalised partial outputs
   float2* part_ml;         // [slot][256] (running max in the log2 domain, row sum)
+  float* part_mid;         // [slot][256] Spatial proxy only: the part of the row sum that came from the middle blocks
   float* f32_o;            // [pass][L][H][d] normalised fp32 outputs (classification)
   float* f32_lse;          // [pass][L][H] natural-log LSE; Spatial proxy also writes [pass + 1] = middle-block LSE
   int32_t n_heads, tokens_per_frame, grid_w, block_tokens;
@@ -499,6 +500,7 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const AttnParams 
       if (row_valid && half == 0) {
         if (w.out_mode == OUT_PARTIAL) {
           p.part_ml[static_cast<size_t>(w.out_slot) * 256 + t * 128 + r] = make_float2(m_ref, l_sum);
+          if (PROXY) p.part_mid[static_cast<size_t>(w.out_slot) * 256 + t * 128 + r] = l_mid;
         } else if (w.out_mode == OUT_F32_LSE) {
           const float ln2 = 0.6931471805599453f;
           const size_t lh = static_cast<size_t>(p.block_tokens) * p.n_heads;
@@ -629,6 +631,50 @@ cls_combine_kernel(const ClsGroup* groups, const ClsPart* parts, const float* pa
     dst[0] = make_float4(acc[k][0] * inv, acc[k][1] * inv, acc[k][2] * inv, acc[k][3] * inv);
     dst[1] = make_float4(acc[k][4] * inv, acc[k][5] * inv, acc[k][6] * inv, acc[k][7] * inv);
     if (c == 0) f32_lse[k * lh + idx] = (l[k] > 0.f) ? m[k] * ln2 + __logf(l[k]) : -INFINITY;
+  }
+}
+
+// Classification, Spatial proxy: the band of one query pair may be cut into pieces along its key range like any other
+// item; this merges the pieces into the proxy output (pass `pass`), its log-sum-exp (plane `pass`) and the
+// log-sum-exp of the middle blocks' share (plane `pass` + 1).
+template <int D>
+__global__ void __launch_bounds__(COMBINE_ROWS * (D / 8))
+proxy_combine_kernel(const ClsGroup* groups, const ClsPart* parts, const float* part_o, const float2* part_ml,
+                     const float* part_mid, float* f32_o, float* f32_lse, int n_heads, int block_tokens, int pass) {
+  constexpr int CHUNKS = D / 8;
+  constexpr int BLOCKS_PER_TILE = 128 / COMBINE_ROWS;
+  const ClsGroup g = groups[blockIdx.x / (2 * BLOCKS_PER_TILE)];
+  const int sub = (blockIdx.x / BLOCKS_PER_TILE) & 1;
+  const int r = (blockIdx.x % BLOCKS_PER_TILE) * COMBINE_ROWS + threadIdx.x / CHUNKS;
+  const int c = threadIdx.x % CHUNKS;
+  if (r >= g.q_count[sub] || g.n_parts == 0) return;  // a band left whole has written its output itself
+  const ClsPart* pp = parts + g.first_part;
+  float m = -INFINITY;
+  for (int i = 0; i < g.n_parts; ++i) m = fmaxf(m, part_ml[static_cast<size_t>(pp[i].slot) * 256 + sub * 128 + r].x);
+  float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0}, l = 0.f, l_mid = 0.f;
+  for (int i = 0; i < g.n_parts; ++i) {
+    const size_t row = static_cast<size_t>(pp[i].slot) * 256 + sub * 128 + r;
+    const float2 ml = part_ml[row];
+    if (ml.x == -INFINITY) continue;
+    const float wgt = ex2_approx(ml.x - m);
+    l += wgt * ml.y;
+    l_mid += wgt * part_mid[row];
+    const float4* src = reinterpret_cast<const float4*>(part_o + row * D + c * 8);
+    const float4 a = src[0], b = src[1];
+    acc[0] += wgt * a.x; acc[1] += wgt * a.y; acc[2] += wgt * a.z; acc[3] += wgt * a.w;
+    acc[4] += wgt * b.x; acc[5] += wgt * b.y; acc[6] += wgt * b.z; acc[7] += wgt * b.w;
+  }
+  const int token = g.q_start + sub * 128 + r;
+  const size_t lh = static_cast<size_t>(block_tokens) * n_heads;
+  const size_t idx = static_cast<size_t>(token) * n_heads + g.head;
+  const float ln2 = 0.6931471805599453f;
+  const float inv = l > 0.f ? 1.f / l : 0.f;
+  float4* dst = reinterpret_cast<float4*>(f32_o + (pass * lh + idx) * D + c * 8);
+  dst[0] = make_float4(acc[0] * inv, acc[1] * inv, acc[2] * inv, acc[3] * inv);
+  dst[1] = make_float4(acc[4] * inv, acc[5] * inv, acc[6] * inv, acc[7] * inv);
+  if (c == 0) {
+    f32_lse[pass * lh + idx] = (l > 0.f) ? m * ln2 + __logf(l) : -INFINITY;
+    f32_lse[(pass + 1) * lh + idx] = (l_mid > 0.f) ? m * ln2 + __logf(l_mid) : -INFINITY;
   }
 }
 

@@ -103,6 +103,7 @@ struct headcast_ctx {
   cudaEvent_t ev_host[8] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
   DevBuf<float> part_o;
   DevBuf<float2> part_ml;
+  DevBuf<float> part_mid;
   DevBuf<float> cls_o, cls_lse, cls_tok, cls_scores;
   DevBuf<int32_t> cls_labels;
 
@@ -198,6 +199,7 @@ struct Proto {  // one (head, query-tile pair, key range) before it is cut into 
   int n_tiles;
   int cls_group = -1;  // classification: every piece writes a partial result that belongs to this group ...
   int cls_tag = 0;     // ... with this tag (0 first block, 1 middle blocks, 2 newest block)
+  bool whole_is_final = false;  // ... unless the item stays in one piece, which then writes its own output mode
 };
 
 void add_query_pairs(std::vector<Proto>& out, WorkItem base, int n_queries, int n_tiles) {
@@ -313,13 +315,13 @@ void finalize_schedule(headcast_ctx* c, Schedule& s, std::vector<Proto>& protos,
           w.tile_begin = begin;
           w.tile_end = begin + take;
           parts.push_back(std::make_pair(cta, w));
-          const bool cut = (take < left) || begin > 0 || p.cls_group >= 0;
+          const bool cut = (take < left) || begin > 0 || (p.cls_group >= 0 && !p.whole_is_final);
           const double cost = per_tile * take + overhead + (cut ? PARTIAL_EXTRA : 0.0);
           room -= cost;
           if (cta == n_cta - 1) last_load += cost;
           begin += take;
         }
-        if (p.cls_group >= 0) {
+        if (p.cls_group >= 0 && !(p.whole_is_final && parts.size() == 1)) {
           for (auto& pr : parts) {
             pr.second.out_mode = OUT_PARTIAL;
             pr.second.out_slot = s.n_slots++;
@@ -566,6 +568,7 @@ int upload_schedule(headcast_ctx* c, Schedule& s, cudaStream_t st) {
   if (s.n_slots > 0) {
     HC_CUDA(c, c->part_o.reserve(static_cast<size_t>(s.n_slots) * 256 * c->D));
     HC_CUDA(c, c->part_ml.reserve(static_cast<size_t>(s.n_slots) * 256));
+    HC_CUDA(c, c->part_mid.reserve(static_cast<size_t>(s.n_slots) * 256));
   }
   s.uploaded = true;
   return HC_OK;
@@ -604,6 +607,7 @@ int run_schedule(headcast_ctx* c, Schedule& s, const void* q, void* out, bool pr
   p.out = static_cast<__nv_bfloat16*>(out);
   p.part_o = c->part_o.ptr;
   p.part_ml = c->part_ml.ptr;
+  p.part_mid = c->part_mid.ptr;
   p.f32_o = c->cls_o.ptr;
   p.f32_lse = c->cls_lse.ptr;
   p.n_heads = c->H;
@@ -635,7 +639,19 @@ int run_schedule(headcast_ctx* c, Schedule& s, const void* q, void* out, bool pr
   else
     rc = proxy ? launch_attn_t<64, true>(c, p, st) : launch_attn_t<64, false>(c, p, st);
   if (rc != HC_OK) return rc;
-  if (!s.cls_groups.empty()) {
+  if (!s.cls_groups.empty() && proxy) {
+    const unsigned blocks = static_cast<unsigned>(s.cls_groups.size()) * 2 * (128 / COMBINE_ROWS);
+    if (c->D == 128)
+      proxy_combine_kernel<128><<<blocks, COMBINE_ROWS * 16, 0, st>>>(s.cls_groups_dev.ptr, s.cls_parts_dev.ptr, c->part_o.ptr,
+                                                                      c->part_ml.ptr, c->part_mid.ptr, c->cls_o.ptr,
+                                                                      c->cls_lse.ptr, c->H, c->L, 3);
+    else
+      proxy_combine_kernel<64><<<blocks, COMBINE_ROWS * 8, 0, st>>>(s.cls_groups_dev.ptr, s.cls_parts_dev.ptr, c->part_o.ptr,
+                                                                    c->part_ml.ptr, c->part_mid.ptr, c->cls_o.ptr,
+                                                                    c->cls_lse.ptr, c->H, c->L, 3);
+    HC_CUDA(c, cudaGetLastError());
+    ++c->launches;
+  } else if (!s.cls_groups.empty()) {
     const unsigned blocks = static_cast<unsigned>(s.cls_groups.size()) * 2 * (128 / COMBINE_ROWS);
     if (c->D == 128)
       cls_combine_kernel<128><<<blocks, COMBINE_ROWS * 16, 0, st>>>(s.cls_groups_dev.ptr, s.cls_parts_dev.ptr, c->part_o.ptr,
@@ -906,6 +922,7 @@ int headcast_destroy(headcast_ctx* c) {
     if (e) cudaEventDestroy(e);
   c->part_o.release();
   c->part_ml.release();
+  c->part_mid.release();
   c->trace_dev.release();
   c->cls_o.release();
   c->cls_lse.release();
@@ -1063,6 +1080,7 @@ int headcast_classify(headcast_ctx* c, const void* q, int32_t* labels_host, floa
   if (c->sched_proxy.key_filled != cls_key) {
     // Spatial proxy: per query-tile pair, the band of grid rows within r of any of its queries, in every cached frame
     std::vector<Proto> protos;
+    c->sched_proxy.cls_groups.clear();
     const int r = c->cfg.proxy_radius;
     for (int h = 0; h < c->H; ++h)
       for (int q0 = 0; q0 < c->L; q0 += 256) {
@@ -1086,9 +1104,21 @@ int headcast_classify(headcast_ctx* c, const void* q, int32_t* labels_host, floa
         p.n_tiles = w.tiles_per_seg * n_filled(c) * c->F_b;
         p.w.tile_begin = 0;
         p.w.tile_end = p.n_tiles;
+        // a band cut into pieces writes partial results, which proxy_combine_kernel merges
+        ClsGroup g;
+        g.head = h;
+        g.q_start = q0;
+        g.q_count[0] = p.w.q_count[0];
+        g.q_count[1] = p.w.q_count[1];
+        g.first_part = 0;
+        g.n_parts = 0;
+        p.cls_group = static_cast<int>(c->sched_proxy.cls_groups.size());
+        p.cls_tag = 0;
+        p.whole_is_final = true;
+        c->sched_proxy.cls_groups.push_back(g);
         protos.push_back(p);
       }
-    finalize_schedule(c, c->sched_proxy, protos, false);
+    finalize_schedule(c, c->sched_proxy, protos, true);
     c->sched_proxy.key_filled = cls_key;
   }
   rc = run_schedule(c, c->sched_proxy, q, nullptr, true, st);
