@@ -304,6 +304,76 @@ def run_rollout(args):
     }))
 
 
+def run_sharded(args, w):
+    """Opt-in (`--shard heads`): ONE layer's heads spread over the ranks (paper_2607_20125_b200/sharding.py) instead of
+    the default of one independent replica per GPU.  Every rank holds Q / K / V in full, attends its own heads and the
+    outputs are all-gathered; total work is fixed, so the scaling is strong.  Prints the same metric as the default
+    run, without the one-time phases."""
+    import torch
+    import torch.distributed as dist
+    from paper_2607_20125_b200 import sharding
+
+    rank, world = int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    else:  # a group of one rank, so that the same code path runs on one GPU
+        dist.init_process_group("gloo", init_method="tcp://127.0.0.1:%d" % (29500 + os.getpid() % 2000), rank=0, world_size=1)
+    L, H, D = w.block_tokens, w.n_heads, w.head_dim
+    n_cells = -(-w.grid_h // w.cell_h) * -(-w.grid_w // w.cell_w)
+    flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    layer = sharding.HeadShardedHeadCast(H, D, L, n_cells, grid_h=w.grid_h, grid_w=w.grid_w, n_blocks=w.n_blocks,
+                                         frames_per_block=w.frames_per_block, cell_h=w.cell_h, cell_w=w.cell_w,
+                                         sd_mode=args.sd_mode, sd_blocks=1 + args.sd_mode)
+    n_extra = 3
+    kv = [tuple(to_dev(t, torch) for t in synth.make_kv(w, b)) for b in range(w.n_blocks + n_extra)]
+    qs = [[to_dev(synth.make_q(w, w.n_blocks + e, s), torch) for s in range(STEPS_PER_BLOCK)] for e in range(n_extra)]
+    out = torch.empty_like(qs[0][0])
+    for b in range(w.n_blocks):
+        layer.append(*kv[b])
+    layer.split_cache(w.labels)  # the planted labels; heads are re-dealt by cost and the moved caches exchanged
+    state = {"i": 0}
+
+    def step():
+        i = state["i"]
+        e = (i // STEPS_PER_BLOCK) % n_extra
+        if i % STEPS_PER_BLOCK == 0:
+            layer.append(*kv[w.n_blocks + e])
+        layer.attend(qs[e][i % STEPS_PER_BLOCK], out)
+        state["i"] = i + 1
+
+    for _ in range(args.warmup):
+        step()
+    times = []
+    torch.cuda.synchronize()
+    dist.barrier()
+    with ClockSampler(local) as sampler:
+        for _ in range(args.steps):
+            flush_buf.zero_()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            step()
+            b.record()
+            b.synchronize()
+            times.append(a.elapsed_time(b))
+        torch.cuda.synchronize()
+        dist.barrier()
+    clocks = sampler.summary()
+    ms = max_over_ranks(float(np.mean(times)), dist if world > 1 else None, torch, "cuda")
+    owner = layer.owner_heads
+    dist.destroy_process_group()
+    if rank != 0:
+        return
+    print(json.dumps({
+        "metric": METRIC, "value": ms, "unit": "ms", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": False, "scaling": "strong", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": args.workload, "parallelism": "heads/%d" % world, "heads_per_rank": [len(h) for h in owner],
+                   "l2": "flushed between steps", "exchange": "all-gather of L x H x d bf16 per attend"},
+        "clocks": clocks, "gpu_launches": None, "e2e": None, "roofline": None, "cpu_baseline": None}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -323,6 +393,8 @@ def main():
                     help="rollout: also replay the steady-state blocks from CUDA graphs (one per layer and ring position)")
     ap.add_argument("--ablations", action="store_true",
                     help="single layer: also time headcast_attend for the label sets of the paper's archetype ablation")
+    ap.add_argument("--shard", default="none", choices=["none", "heads"],
+                    help="heads: one layer's heads spread over the ranks (strong scaling) instead of one replica per GPU")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-phases", action="store_true")
     args = ap.parse_args()
@@ -335,6 +407,8 @@ def main():
     w = workload_of(args.workload)
     if args.impl == "reference":
         return run_reference(args, w)
+    if args.shard == "heads":
+        return run_sharded(args, w)
 
     import torch
     from paper_2607_20125_b200.binding import HeadCast

@@ -247,15 +247,21 @@ class HeadCast:
         """q_host / out_host: CPU tensors (pinned for overlap); out_host is complete after the stream is synchronised."""
         self._check(self.lib.headcast_attend_host(self._ctx, _host_ptr(q_host), _host_ptr(out_host), _stream()))
 
-    def export_cache(self, head: int):
-        """Returns (K, V) uint16 CPU arrays [n_tokens, d] of what the cache keeps for ``head``."""
+    def export_cache_device(self, head: int):
+        """Returns (K, V) bf16 device tensors [n_tokens, d] of what the cache keeps for ``head``, logical order."""
         import torch
         n = C.c_int32()
         k = torch.empty((self.n_blocks * self.block_tokens, self.head_dim), dtype=torch.bfloat16, device="cuda")
         v = torch.empty_like(k)
         self._check(self.lib.headcast_export_cache(self._ctx, head, _ptr(k), _ptr(v), C.byref(n), _stream()))
         torch.cuda.current_stream().synchronize()
-        to_bits = lambda t: t[: n.value].view(torch.int16).cpu().numpy().view("uint16")
+        return k[: n.value], v[: n.value]
+
+    def export_cache(self, head: int):
+        """Returns (K, V) uint16 CPU arrays [n_tokens, d] of what the cache keeps for ``head``."""
+        import torch
+        k, v = self.export_cache_device(head)
+        to_bits = lambda t: t.view(torch.int16).cpu().numpy().view("uint16")
         return to_bits(k), to_bits(v)
 
     def n_filled(self) -> int:
