@@ -137,17 +137,18 @@ def test_random_geometries(gh, gw, ch, cw, n_blocks, fill, heads, n_ctas, d):
     check_plan(w, heads, min(fill, n_blocks), n_ctas)
 
 
-@settings(max_examples=25, deadline=None)
+@settings(max_examples=40, deadline=None)
 @given(gh=st.integers(20, 70), gw=st.integers(30, 120), n_blocks=st.integers(3, 8),
        heads=st.lists(st.integers(0, 3), min_size=6, max_size=16), n_ctas=st.sampled_from([37, 148, 160]))
-def test_large_workloads_use_nearly_every_cta(gh, gw, n_blocks, heads, n_ctas):
-    """Whatever the grid and the head mix, a workload much larger than the machine must not leave a noticeable share
-    of the CTAs without work (the share search falls back to an upward scan when its bisection goes astray)."""
+def test_large_workloads_are_spread_evenly(gh, gw, n_blocks, heads, n_ctas):
+    """Whatever the grid and the head mix, a workload much larger than the machine is spread evenly: no CTA carries
+    much more than the mean (the share search falls back to an upward scan when its bisection goes astray)."""
     w = synth.Workload("big", len(heads), 128, gh, gw, n_blocks, labels=tuple(heads))
     items, per_cta = check_plan(w, heads, n_blocks, n_ctas)
     if per_cta.sum() > 40.0 * n_ctas:  # several items' worth of work per CTA
-        assert (per_cta == 0).sum() <= max(2, n_ctas // 20), ((per_cta == 0).sum(), per_cta.mean())
-        assert per_cta.max() <= 1.15 * per_cta.mean()
+        # the busiest CTA decides the launch: it may not carry much more than an equal share (whole items of about
+        # half a share cannot be dealt more evenly without paying for cuts, hence the slack; some CTAs may then idle)
+        assert per_cta.max() <= 1.15 * per_cta.mean(), (per_cta.max(), per_cta.mean(), (per_cta == 0).sum())
 
 
 def test_planner_rejects_bad_input():
