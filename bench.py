@@ -573,7 +573,7 @@ def main():
 
     # ---- end to end: the host-buffer entry points of the C ABI (pinned host tensors), every copy inside the timed
     # region: headcast_append_host every 4th step, headcast_attend_host (query columns in, outputs out, overlapped
-    # with the kernels group by group), stream synchronised before the clock stops
+    # with the kernels stage by stage), stream synchronised before the clock stops
     host_q = [q.cpu().pin_memory() for q in q_extra[0]]
     host_kv = [(k.cpu().pin_memory(), v.cpu().pin_memory()) for k, v in kv[w.n_blocks:w.n_blocks + 2]]
     host_out = torch.empty_like(host_q[0]).pin_memory()

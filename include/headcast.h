@@ -157,9 +157,10 @@ int64_t headcast_launch_count(const headcast_ctx* ctx);
  * is for measuring, or serving, the path end to end across PCIe).  k_host/v_host/q_host/out_host: host pointers to
  * [L][H][d] bf16; pinned memory lets the copies overlap the kernels, pageable memory works but serialises.
  * headcast_append_host copies the block into device staging owned by the context and appends it.
- * headcast_attend_host splits the call by archetype group (Global, Spatial, Sink + Dummy heads): each group's query
- * columns are copied in, attended (Sec. 4.4, as headcast_attend) and its output columns copied out, on two copy
- * streams of the context, so that transfers in both directions overlap the attention of the other groups.  Both
+ * headcast_attend_host splits the call into four stages (first half of the Global heads' query rows; Sink + Dummy
+ * heads; Spatial heads; second half of the Global heads' rows): each stage's part of Q is copied in, attended
+ * (Sec. 4.4, as headcast_attend) and its part of the output copied out, on two copy streams of the context, so that
+ * transfers in both directions overlap the attention of the other stages.  Both
  * return once everything is enqueued; out_host is complete when work enqueued on `stream` after the call runs (e.g.
  * after synchronising `stream`).  q_host must stay unchanged and out_host untouched until then.  Staging buffers,
  * streams and events are created on the first call.  Errors as headcast_attend / headcast_append. */

@@ -97,10 +97,13 @@ struct headcast_ctx {
   int32_t* status_dev = nullptr;
 
   Schedule sched_dense, sched_hc, sched_cls, sched_proxy;
-  Schedule sched_group[3];  // headcast_attend_host: Global / Spatial / Sink+Dummy heads on their own
+  // headcast_attend_host: the stages of its pipeline, each with its own work list - the first half of the Global
+  // heads' rows, the Sink + Dummy heads, the Spatial heads, the second half of the Global heads' rows
+  static constexpr int N_HOST_STAGES = 4;
+  Schedule sched_stage[N_HOST_STAGES];
   DevBuf<__nv_bfloat16> stage_q, stage_out, stage_k, stage_v;  // device copies of host tensors
   cudaStream_t copy_in = nullptr, copy_out = nullptr;
-  cudaEvent_t ev_host[8] = {nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr};
+  cudaEvent_t ev_host[2 + 2 * N_HOST_STAGES] = {};
   DevBuf<float> part_o;
   DevBuf<float2> part_ml;
   DevBuf<float> part_mid;
@@ -202,8 +205,10 @@ struct Proto {  // one (head, query-tile pair, key range) before it is cut into 
   bool whole_is_final = false;  // ... unless the item stays in one piece, which then writes its own output mode
 };
 
-void add_query_pairs(std::vector<Proto>& out, WorkItem base, int n_queries, int n_tiles) {
-  for (int q0 = 0; q0 < n_queries; q0 += 256) {
+// Query-tile pairs of rows [q_lo, q_hi) (q_lo a multiple of 256; by default all rows) of one head and key range.
+void add_query_pairs(std::vector<Proto>& out, WorkItem base, int n_queries, int n_tiles, int q_lo = 0, int q_hi = -1) {
+  const int q_end = (q_hi < 0) ? n_queries : std::min(q_hi, n_queries);
+  for (int q0 = q_lo; q0 < q_end; q0 += 256) {
     Proto p;
     p.w = base;
     p.w.q_start[0] = q0;
@@ -508,7 +513,9 @@ void build_dense_schedule(headcast_ctx* c, Schedule& s, int out_mode, bool allow
 }
 
 // group < 0: every head; 0: Global heads only; 1: Spatial; 2: Sink and Dummy
-void build_headcast_schedule(headcast_ctx* c, Schedule& s, int group = -1) {
+// group < 0: every head; else only the heads of one archetype group (0 Global, 1 Spatial, 2 Sink + Dummy), and for
+// groups 0 and 2 only the query rows [q_lo, q_hi) (q_lo a multiple of 256; q_hi < 0: to the end).
+void build_headcast_schedule(headcast_ctx* c, Schedule& s, int group = -1, int q_lo = 0, int q_hi = -1) {
   std::vector<Proto> protos;
   const int nf = n_filled(c);
   const long long win = static_cast<long long>(c->n_blk) * c->L;
@@ -522,11 +529,11 @@ void build_headcast_schedule(headcast_ctx* c, Schedule& s, int group = -1) {
       long long row0 = static_cast<long long>(j) * c->sd_slots * c->L;
       if (cl == CLS_DUMMY && c->sd_valid == 1) row0 += static_cast<long long>(c->dummy_cur) * c->L;
       WorkItem w = range_item(h, MAP_SD, 0, row0, c->sd_valid * c->L);
-      add_query_pairs(protos, w, c->L, w.tiles_per_seg);
+      add_query_pairs(protos, w, c->L, w.tiles_per_seg, q_lo, q_hi);
       flops += 4.0 * c->L * static_cast<double>(c->sd_valid) * c->L * c->D;
     } else if (cl == CLS_GLOBAL) {
       WorkItem w = range_item(h, MAP_GLOBAL, 0, ix * win, nf * c->L);
-      add_query_pairs(protos, w, c->L, w.tiles_per_seg);
+      add_query_pairs(protos, w, c->L, w.tiles_per_seg, q_lo, q_hi);
       flops += 4.0 * c->L * static_cast<double>(nf) * c->L * c->D;
     } else {
       for (size_t ci = 0; ci < c->cells.size(); ++ci) {
@@ -911,7 +918,7 @@ int headcast_destroy(headcast_ctx* c) {
   c->sched_hc.release();
   c->sched_cls.release();
   c->sched_proxy.release();
-  for (Schedule& g : c->sched_group) g.release();
+  for (Schedule& g : c->sched_stage) g.release();
   c->stage_q.release();
   c->stage_out.release();
   c->stage_k.release();
@@ -1258,28 +1265,37 @@ int headcast_attend_host(headcast_ctx* c, const void* q_host, void* out_host, vo
   HC_CUDA(c, c->stage_q.reserve(elems));
   HC_CUDA(c, c->stage_out.reserve(elems));
   const int key = n_filled(c) * 4 + c->sd_valid;
-  for (int g = 0; g < 3; ++g)
-    if (c->sched_group[g].key_filled != key) build_headcast_schedule(c, c->sched_group[g], g);
-  // The heads of one archetype group are copied in (strided: the rows of [L][H][d] hold all heads), attended and copied
-  // out as a unit, so that the next group's queries arrive and the previous group's outputs leave while this group
-  // computes.  Global heads go first: most arithmetic per byte moved.
+  // Stages: a stage's queries are copied in (strided: the rows of [L][H][d] hold all heads), attended and copied out
+  // as a unit, so that the next stage's queries arrive and the previous stage's outputs leave while this stage
+  // computes.  The Global heads do most of the arithmetic per byte moved, so their query rows are halved (at a
+  // multiple of 256 rows: the query-tile pairs stay the same) and the halves go first and last: the kernels start
+  // after a small copy, and when they end only a small copy is left; the other heads' copies hide in between.
+  const int mid = ((c->L / 2 + 255) / 256) * 256;
+  struct Stage { int group, lo, hi; };
+  const Stage stages[headcast_ctx::N_HOST_STAGES] = {{0, 0, mid}, {2, 0, c->L}, {1, 0, c->L}, {0, mid, c->L}};
+  for (int i = 0; i < headcast_ctx::N_HOST_STAGES; ++i)
+    if (c->sched_stage[i].key_filled != key)
+      build_headcast_schedule(c, c->sched_stage[i], stages[i].group, stages[i].lo, stages[i].hi);
   const size_t pitch = static_cast<size_t>(c->H) * c->D * sizeof(__nv_bfloat16);
-  auto copy_group = [&](int g, bool in) -> int {
+  auto copy_stage = [&](const Stage& sg, bool in) -> int {
+    const int rows = sg.hi - sg.lo;
+    if (rows <= 0) return HC_OK;
     for (int h0 = 0; h0 < c->H;) {
       auto group_of = [&](int h) { return c->cls[h] == CLS_GLOBAL ? 0 : c->cls[h] == CLS_SPATIAL ? 1 : 2; };
-      if (group_of(h0) != g) {
+      if (group_of(h0) != sg.group) {
         ++h0;
         continue;
       }
       int h1 = h0 + 1;
-      while (h1 < c->H && group_of(h1) == g) ++h1;
-      const size_t off = static_cast<size_t>(h0) * c->D, width = static_cast<size_t>(h1 - h0) * c->D * sizeof(__nv_bfloat16);
+      while (h1 < c->H && group_of(h1) == sg.group) ++h1;
+      const size_t off = static_cast<size_t>(sg.lo) * c->H * c->D + static_cast<size_t>(h0) * c->D;
+      const size_t width = static_cast<size_t>(h1 - h0) * c->D * sizeof(__nv_bfloat16);
       if (in)
         HC_CUDA(c, cudaMemcpy2DAsync(c->stage_q.ptr + off, pitch, static_cast<const __nv_bfloat16*>(q_host) + off, pitch, width,
-                                     c->L, cudaMemcpyHostToDevice, c->copy_in));
+                                     rows, cudaMemcpyHostToDevice, c->copy_in));
       else
         HC_CUDA(c, cudaMemcpy2DAsync(static_cast<__nv_bfloat16*>(out_host) + off, pitch, c->stage_out.ptr + off, pitch, width,
-                                     c->L, cudaMemcpyDeviceToHost, c->copy_out));
+                                     rows, cudaMemcpyDeviceToHost, c->copy_out));
       h0 = h1;
     }
     return HC_OK;
@@ -1288,18 +1304,18 @@ int headcast_attend_host(headcast_ctx* c, const void* q_host, void* out_host, vo
   HC_CUDA(c, cudaEventRecord(c->ev_host[0], st));
   HC_CUDA(c, cudaStreamWaitEvent(c->copy_in, c->ev_host[0], 0));
   HC_CUDA(c, cudaStreamWaitEvent(c->copy_out, c->ev_host[0], 0));
-  for (int g = 0; g < 3; ++g) {
-    if (c->sched_group[g].items.empty()) continue;
-    if ((rc = copy_group(g, true)) != HC_OK) return rc;
-    HC_CUDA(c, cudaEventRecord(c->ev_host[1 + g], c->copy_in));
-    HC_CUDA(c, cudaStreamWaitEvent(st, c->ev_host[1 + g], 0));
-    if ((rc = run_schedule(c, c->sched_group[g], c->stage_q.ptr, c->stage_out.ptr, false, st)) != HC_OK) return rc;
-    HC_CUDA(c, cudaEventRecord(c->ev_host[4 + g], st));
-    HC_CUDA(c, cudaStreamWaitEvent(c->copy_out, c->ev_host[4 + g], 0));
-    if ((rc = copy_group(g, false)) != HC_OK) return rc;
+  for (int i = 0; i < headcast_ctx::N_HOST_STAGES; ++i) {
+    if (c->sched_stage[i].items.empty()) continue;
+    if ((rc = copy_stage(stages[i], true)) != HC_OK) return rc;
+    HC_CUDA(c, cudaEventRecord(c->ev_host[2 + 2 * i], c->copy_in));
+    HC_CUDA(c, cudaStreamWaitEvent(st, c->ev_host[2 + 2 * i], 0));
+    if ((rc = run_schedule(c, c->sched_stage[i], c->stage_q.ptr, c->stage_out.ptr, false, st)) != HC_OK) return rc;
+    HC_CUDA(c, cudaEventRecord(c->ev_host[3 + 2 * i], st));
+    HC_CUDA(c, cudaStreamWaitEvent(c->copy_out, c->ev_host[3 + 2 * i], 0));
+    if ((rc = copy_stage(stages[i], false)) != HC_OK) return rc;
   }
-  HC_CUDA(c, cudaEventRecord(c->ev_host[7], c->copy_out));
-  HC_CUDA(c, cudaStreamWaitEvent(st, c->ev_host[7], 0));
+  HC_CUDA(c, cudaEventRecord(c->ev_host[1], c->copy_out));
+  HC_CUDA(c, cudaStreamWaitEvent(st, c->ev_host[1], 0));
   return HC_OK;
 }
 
