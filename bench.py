@@ -31,7 +31,7 @@ METRIC = "headcast_attn_ms_per_block_step"
 STEPS_PER_BLOCK = 4
 # dram__bytes_read.sum + dram__bytes_write.sum of one attention-kernel launch, from the ncu captures summarised
 # under profiles/ (None where not captured at that size)
-NCU_TRAFFIC_BYTES = {"480p": 379.3e6, "720p": 580.5e6, "1080p": None, "tiny": None}
+NCU_TRAFFIC_BYTES = {"480p": 279.0e6, "720p": 606.0e6, "1080p": None, "tiny": None}
 
 
 def workload_of(name: str):

@@ -84,6 +84,9 @@ constexpr int KV_SLOTS = 4;  // one shared-memory ring for K and V tiles, filled
 #ifndef HC_POLY_MASK
 #define HC_POLY_MASK 3  // pairs whose index has all these bits set take the polynomial exponential (3: every 4th)
 #endif
+#ifndef HC_L2_HINT
+#define HC_L2_HINT 2  // 1: Spatial cells' K/V are loaded evict-first; 2: the other K/V also evict-last
+#endif
 #ifndef HC_RESCALE_THRESHOLD
 #define HC_RESCALE_THRESHOLD 8.0f
 #endif
@@ -192,10 +195,19 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const AttnParams 
     if (lane == 0) {
       uint32_t kt = 0;
       bool ok = true;
+      // L2 policy per item: a Spatial cell's keys are read by one item only (its queries fill at most one tile pair),
+      // so they stream through L2 without pushing out the long K/V streams that every query tile of a head re-reads
+      const uint64_t pol_stream = l2_policy_evict_first();
+#if HC_L2_HINT == 2
+      const uint64_t pol_keep = l2_policy_evict_last();
+#else
+      const uint64_t pol_keep = l2_policy_evict_normal();
+#endif
       for (int it = item_lo; it < item_hi && ok; ++it) {
         const WorkItem w = p.items[it];
         const CUtensorMap* kmap = &p.maps[2 * w.kv_map];
         const CUtensorMap* vmap = kmap + 1;
+        const uint64_t policy = (HC_L2_HINT && w.cell >= 0) ? pol_stream : pol_keep;
         for (int tile = w.tile_begin; tile < w.tile_end; ++tile, ++kt) {
           const int seg = tile / w.tiles_per_seg, c = tile - seg * w.tiles_per_seg;
           const int row = w.kv_row0 + seg * w.seg_stride + c * 128;
@@ -205,8 +217,8 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const AttnParams 
             if (!(ok = mbar_wait(&bar_kv_free[st], ph ^ 1, abortp, p.status, 11 + kv))) break;
             mbar_arrive_expect_tx(&bar_kv_full[st], SM::TILE_BYTES);
             for (int b = 0; b < NB; ++b)
-              tma_load_2d(smem + SM::KV_OFF + st * SM::TILE_BYTES + b * SM::BLOCK_BYTES, kv ? vmap : kmap,
-                          w.kv_x0 + 64 * b, row, &bar_kv_full[st]);
+              tma_load_2d_hint(smem + SM::KV_OFF + st * SM::TILE_BYTES + b * SM::BLOCK_BYTES, kv ? vmap : kmap,
+                               w.kv_x0 + 64 * b, row, &bar_kv_full[st], policy);
           }
           if (!ok) break;
         }
