@@ -91,14 +91,16 @@ __device__ float block_select(const float* v, int n, int k, uint32_t* hist /* [2
       if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
     }
     __syncthreads();
-    if (threadIdx.x == 0) {
-      int acc = 0, digit = 0;
-      for (; digit < 256; ++digit) {
-        if (acc + static_cast<int>(hist[digit]) > remaining) break;
-        acc += hist[digit];
+    if (threadIdx.x < 256) {
+      // the digit whose bin holds rank `remaining`: thread d adds up the bins below d (all threads read the same bin
+      // at the same time: a broadcast), exactly one thread finds the rank inside its own bin
+      uint32_t below = 0;
+      for (int d = 0; d < static_cast<int>(threadIdx.x); ++d) below += hist[d];
+      const uint32_t rank = static_cast<uint32_t>(remaining);
+      if (below <= rank && rank < below + hist[threadIdx.x]) {
+        bcast[0] = threadIdx.x;
+        bcast[1] = rank - below;
       }
-      bcast[0] = static_cast<uint32_t>(digit);
-      bcast[1] = static_cast<uint32_t>(remaining - acc);
     }
     __syncthreads();
     prefix |= bcast[0] << shift;
@@ -121,23 +123,34 @@ struct DecideParams {
 
 // One block per head: fixed-order sums (deterministic), percentile by selection, Eq. 4 and Eq. 5.
 __global__ void __launch_bounds__(512) head_decide_kernel(const DecideParams p) {
-  __shared__ double red[512];
+  __shared__ double red[TOK_N][16];
   __shared__ uint32_t hist[256];
   __shared__ uint32_t bcast[2];
   __shared__ double sums[TOK_N];
   const int h = blockIdx.x;
   const size_t hl = static_cast<size_t>(p.H) * p.L;
-  for (int q = 0; q < TOK_N; ++q) {
-    const float* v = p.tok + q * hl + static_cast<size_t>(h) * p.L;
-    double acc = 0.0;
-    for (int i = threadIdx.x; i < p.L; i += blockDim.x) acc += static_cast<double>(v[i]);
-    red[threadIdx.x] = acc;
-    __syncthreads();
-    for (int s = blockDim.x / 2; s > 0; s >>= 1) {
-      if (threadIdx.x < s) red[threadIdx.x] += red[threadIdx.x + s];
-      __syncthreads();
+  {
+    // all per-token quantities in one pass; the order of every sum is fixed by the thread layout alone
+    double acc[TOK_N];
+#pragma unroll
+    for (int q = 0; q < TOK_N; ++q) acc[q] = 0.0;
+    const float* v = p.tok + static_cast<size_t>(h) * p.L;
+    for (int i = threadIdx.x; i < p.L; i += blockDim.x) {
+#pragma unroll
+      for (int q = 0; q < TOK_N; ++q) acc[q] += static_cast<double>(v[q * hl + i]);
     }
-    if (threadIdx.x == 0) sums[q] = red[0];
+#pragma unroll
+    for (int q = 0; q < TOK_N; ++q) {
+      double x = acc[q];
+      for (int off = 16; off > 0; off >>= 1) x += __shfl_down_sync(0xffffffffu, x, off);
+      if ((threadIdx.x & 31) == 0) red[q][threadIdx.x >> 5] = x;
+    }
+    __syncthreads();
+    if (threadIdx.x < TOK_N) {
+      double x = 0.0;
+      for (int wp = 0; wp < static_cast<int>(blockDim.x >> 5); ++wp) x += red[threadIdx.x][wp];
+      sums[threadIdx.x] = x;
+    }
     __syncthreads();
   }
   const float* cos_sp = p.tok + TOK_COS_SPATIAL * hl + static_cast<size_t>(h) * p.L;
