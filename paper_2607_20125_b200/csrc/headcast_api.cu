@@ -1270,7 +1270,7 @@ int headcast_attend_host(headcast_ctx* c, const void* q_host, void* out_host, vo
   // computes.  The Global heads do most of the arithmetic per byte moved, so their query rows are halved (at a
   // multiple of 256 rows: the query-tile pairs stay the same) and the halves go first and last: the kernels start
   // after a small copy, and when they end only a small copy is left; the other heads' copies hide in between.
-  const int mid = ((c->L / 2 + 255) / 256) * 256;
+  const int mid = std::min(c->L, ((c->L / 2 + 255) / 256) * 256);  // blocks of up to 256 tokens have one stage per group
   struct Stage { int group, lo, hi; };
   const Stage stages[headcast_ctx::N_HOST_STAGES] = {{0, 0, mid}, {2, 0, c->L}, {1, 0, c->L}, {0, mid, c->L}};
   for (int i = 0; i < headcast_ctx::N_HOST_STAGES; ++i)

@@ -367,14 +367,15 @@ def test_refresh_of_the_current_block_in_one_block_mode():
     p.check_attention(dense=True)
 
 
-@pytest.mark.parametrize("labels", [None, [orc.GLOBAL] * 6, [orc.SINK, orc.DUMMY, orc.SPATIAL] * 2])
+@pytest.mark.parametrize("labels", [None, [orc.GLOBAL] * 6, [orc.SINK, orc.DUMMY, orc.SPATIAL] * 2, "tiny"])
 def test_host_buffer_calls_match_the_oracle(labels):
-    """headcast_append_host / headcast_attend_host: host tensors in, host tensor out, group-wise overlap of the
+    """headcast_append_host / headcast_attend_host: host tensors in, host tensor out, stage-wise overlap of the
     copies with the kernels; cache content stays bit-exact and the outputs meet the same bars as headcast_attend.
-    Pinned and pageable host memory are both accepted."""
+    Pinned and pageable host memory are both accepted.  "tiny": a block shorter than one query-tile pair (192
+    tokens), where the Global heads' rows cannot be halved."""
     import torch
-    w = synth.small()
-    lab = w.labels if labels is None else labels
+    w = synth.tiny() if labels == "tiny" else synth.small()
+    lab = w.labels if labels is None or labels == "tiny" else labels
     p = Pair(w)
     p.append(2)
     p.hc.set_labels(lab)
