@@ -423,20 +423,27 @@ def test_seeded_random_shapes(case):
     fill = int(rng.integers(1, w.n_blocks + 1))
     extra = int(rng.integers(1, 2 * w.n_blocks))
     run_pipeline(w, fill=fill, extra=extra, sd_mode=int(rng.integers(0, 2)))
-    # classification of the same shape (needs two cached blocks): scores within the bars; labels must agree wherever
-    # the float64 decision is not within the score tolerance of a threshold
-    cfill = max(2, fill)
-    p = Pair(w)
+    # classification of the same shape (needs two cached blocks; the ring may have rolled), with a drawn proxy radius
+    # and gamma: scores within the bars; labels must agree wherever the float64 decision is not within the score
+    # tolerance of a threshold; the labels found then drive the split
+    r, gamma = int(rng.integers(0, 4)), float(rng.choice([1.0, 5.0, 20.0]))
+    cfill = int(rng.integers(2, 2 * w.n_blocks + 1))
+    p = Pair(w, proxy_radius=r, gamma=gamma)
     p.append(cfill)
     q = synth.make_q(w, cfill - 1, 0)
     labels, scores = p.hc.classify(to_dev(q))
-    want_labels, want = orc.classify(q, p.cache, p.geom)
+    want_labels, want = orc.classify(q, p.cache, p.geom, r=r, gamma=gamma)
     d = np.abs(scores.astype(np.float64) - want)
+    score_tol = 1e-2 + gamma * 2e-3  # score = P5 - gamma * MSE
     assert d[:, [0, 1, 2, 6, 7, 8, 9]].max() <= 5e-3, d
-    assert d[:, [3, 5]].max() <= 1e-2 and d[:, 4].max() <= 2e-3, d
+    assert d[:, 3].max() <= 1e-2 and d[:, 4].max() <= 2e-3 and d[:, 5].max() <= score_tol, d
     theta = np.array([0.95, 0.95, 0.95])
-    decisive = (np.abs(want[:, :3] - theta).min(axis=1) > 1e-2) & (np.abs(want[:, 5] - 0.755) > 2e-2)
+    decisive = (np.abs(want[:, :3] - theta).min(axis=1) > 1e-2) & (np.abs(want[:, 5] - 0.755) > 2 * score_tol)
     assert all(int(a) == int(b) for a, b, ok in zip(labels, want_labels, decisive) if ok), (labels, want_labels)
+    p.hc.split_cache()
+    p.cache.split([int(v) for v in labels])
+    p.check_cache()
+    p.check_attention(dense=False)
 
 
 def test_maximum_head_and_block_counts():
