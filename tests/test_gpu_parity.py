@@ -526,3 +526,91 @@ def test_head_sharded_layer_on_one_rank_equals_the_plain_layer():
     finally:
         if own_group:
             dist.destroy_process_group()
+
+
+def test_two_contexts_on_two_streams_give_the_single_stream_results():
+    # two layers driven from two CUDA streams at once (the library keeps no state outside its contexts): every output
+    # must equal, bit for bit, what the same calls give one after the other
+    import torch
+    from paper_2607_20125_b200.binding import HeadCast
+    ws = [synth.small(seed=synth.BASE_SEED + 5), synth.tiny()]
+
+    def prepare(w):
+        hc = HeadCast.from_workload(w, keep_monolithic=True)
+        for b in range(w.n_blocks):
+            hc.append(*[to_dev(t) for t in synth.make_kv(w, b)])
+        hc.set_labels(w.labels)
+        hc.split_cache()
+        return hc
+
+    def step(hc, w, i, outs):
+        if i % 2 == 0:
+            hc.append(*[to_dev(t) for t in synth.make_kv(w, w.n_blocks + i)])
+        q = to_dev(synth.make_q(w, w.n_blocks + i, i % 4))
+        o = torch.empty_like(q)
+        hc.attend(q, o)
+        outs.append(o)
+
+    ref = [[], []]
+    for i, w in enumerate(ws):
+        hc = prepare(w)
+        for s in range(6):
+            step(hc, w, s, ref[i])
+        torch.cuda.synchronize()
+        hc.check()
+        hc.destroy()
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    got, ctx = [[], []], []
+    for i, w in enumerate(ws):
+        with torch.cuda.stream(streams[i]):
+            ctx.append(prepare(w))
+    for s in range(6):
+        for i, w in enumerate(ws):
+            with torch.cuda.stream(streams[i]):
+                step(ctx[i], w, s, got[i])
+    torch.cuda.synchronize()
+    for i in range(2):
+        ctx[i].check()
+        for a, b in zip(got[i], ref[i]):
+            assert torch.equal(a.view(torch.int16), b.view(torch.int16))
+        ctx[i].destroy()
+
+
+def test_contexts_give_their_device_memory_back():
+    # every phase once per context (dense, classification, split, append, both attends, the host-buffer calls with
+    # their staging buffers, streams and events), 40 contexts in a row: the device memory in use must not grow
+    import torch
+    from paper_2607_20125_b200.binding import HeadCast
+    w = synth.small()
+    kv = [[to_dev(t) for t in synth.make_kv(w, b)] for b in range(w.n_blocks + 1)]
+    q = to_dev(synth.make_q(w, 1, 0))
+    o = torch.empty_like(q)
+    qh, kh, vh = q.cpu().pin_memory(), kv[0][0].cpu().pin_memory(), kv[0][1].cpu().pin_memory()
+    oh = torch.empty_like(qh).pin_memory()
+
+    def once():
+        hc = HeadCast.from_workload(w, keep_monolithic=True)
+        for b in range(w.n_blocks):
+            hc.append(*kv[b])
+        hc.full_attend(q, o)
+        hc.classify(q)
+        hc.split_cache()
+        hc.append(*kv[-1])
+        hc.attend(q, o)
+        hc.append_host(kh, vh)
+        hc.attend_host(qh, oh)
+        torch.cuda.synchronize()
+        hc.check()
+        hc.destroy()
+
+    def in_use():
+        torch.cuda.synchronize()
+        free, total = torch.cuda.mem_get_info()
+        return (total - free) / 2 ** 20
+
+    for _ in range(3):
+        once()
+    before = in_use()
+    for _ in range(40):
+        once()
+    assert in_use() - before < 8.0
