@@ -614,3 +614,31 @@ def test_contexts_give_their_device_memory_back():
     for _ in range(40):
         once()
     assert in_use() - before < 8.0
+
+
+@pytest.mark.parametrize("scale", [0.01, 16.0, 256.0])
+def test_flat_peaked_and_huge_logits(scale):
+    # queries scaled so that the softmax is nearly uniform, nearly one-hot, or has logits in the thousands; a few rows
+    # get one enormous coordinate, so their logits jump by hundreds from one key tile to the next (the running
+    # reference has to be moved and the accumulated output rescaled).  Every pathway, dense and head-specific.
+    import torch
+    w = synth.small()
+    p = Pair(w, sd_mode=1)
+    p.append(w.n_blocks)
+    p.hc.set_labels(w.labels)
+    p.hc.split_cache()
+    p.cache.split(w.labels)
+    rng = np.random.default_rng(99)
+    qf = synth.bf16_bits_to_f32(synth.make_q(w, w.n_blocks - 1, 0)) * scale
+    qf[rng.integers(0, w.block_tokens, size=16), :, 7] *= 50.0
+    q = synth.f32_to_bf16_bits(qf.astype(np.float32))
+    for dense in (True, False):
+        out = torch.full((w.block_tokens, w.n_heads, w.head_dim), float("nan"), dtype=torch.bfloat16, device="cuda")
+        (p.hc.full_attend if dense else p.hc.attend)(to_dev(q), out)
+        p.hc.check()
+        got = to_f64(out)
+        want = orc.full_attend(q, p.cache)[0] if dense else orc.attend(q, p.cache, p.geom)
+        assert np.isfinite(got).all()
+        err = np.abs(got - want)
+        assert (err <= np.maximum(MAX_ABS, np.abs(want) * 2.0 ** -7)).all(), err.max()  # one bf16 step on large outputs
+        assert err.mean(axis=(0, 2)).max() <= MEAN_ABS
