@@ -583,11 +583,15 @@ int upload_schedule(headcast_ctx* c, Schedule& s, cudaStream_t st) {
 
 template <int D, bool PROXY>
 int launch_attn_t(headcast_ctx* c, const AttnParams& p, cudaStream_t st) {
-  static bool configured = false;
-  if (!configured) {
+  // the attribute belongs to the (function, device) pair: one flag per device, so that a process that drives several
+  // GPUs sets it on each of them
+  static bool configured[64] = {};
+  int dev = 0;
+  HC_CUDA(c, cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64 || !configured[dev]) {
     HC_CUDA(c, cudaFuncSetAttribute(attn_kernel<D, PROXY>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                     AttnSmem<D>::DYN_BYTES));
-    configured = true;
+    if (dev >= 0 && dev < 64) configured[dev] = true;
   }
   if (c->timing) HC_CUDA(c, cudaEventRecord(c->ev_a, st));
   attn_kernel<D, PROXY><<<c->n_sm, ATTN_THREADS, AttnSmem<D>::DYN_BYTES, st>>>(p);
