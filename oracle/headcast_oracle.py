@@ -20,7 +20,7 @@ What each function follows:
   Dummy rolling overwrite, Global/Spatial sliding window that keeps the sink block.
 * ``flops_ratio`` / ``kv_reduction`` - the closed forms of Appendix B and C.
 
-Readings taken where the paper is silent (same list as the design notes):
+Readings taken where the paper is silent:
 softmax scale 1/sqrt(d); Sink/Dummy use exactly one block (Sec. 4.4), the
 appendix's "anchor + current block" accounting is only used by the two
 closed-form helpers; cells: n = max(1, floor(G/cell + 1/2)) per axis with edges
@@ -30,7 +30,7 @@ MSE = mean over all L*d elements; cosine denominator clamped at 1e-12.
 
 Parity unpinned (the paper prints no worked example): the percentile
 interpolation rule, the cell rounding rule, and the attention-mass auxiliary
-outputs' "rest" partition.  Everything else is pinned by tests/test_oracle_*.py.
+outputs' "rest" partition.  Everything else is pinned by the CPU test suite.
 """
 from __future__ import annotations
 
@@ -378,13 +378,15 @@ def kv_reduction(n_sink_dummy: float, n_total: float, window: float = 8.0, kept:
     return n_sink_dummy / n_total * (1.0 - kept / window)
 
 
-def attend_flops(geom: Geometry, labels: Sequence[int], n_filled: int, d: int) -> float:
-    """Algorithmic FLOPs (4 * L_q * L_k * d per head, Appendix B) of one head-specific attend."""
+def attend_flops(geom: Geometry, labels: Sequence[int], n_filled: int, d: int, sd_blocks: int = 1) -> float:
+    """Algorithmic FLOPs (4 * L_q * L_k * d per head, Appendix B) of one head-specific attend.
+    ``sd_blocks`` = blocks a Sink / Dummy head reads: 1 (Sec. 4.4) or 2 (the appendix's accounting),
+    never more than are cached."""
     L = geom.block_tokens
     total = 0.0
     for lab in labels:
         if lab in (SINK, DUMMY):
-            total += 4.0 * L * L * d
+            total += 4.0 * L * min(sd_blocks, n_filled) * L * d
         elif lab == GLOBAL:
             total += 4.0 * L * n_filled * L * d
         else:

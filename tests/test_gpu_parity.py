@@ -343,9 +343,7 @@ def test_anchor_plus_current_variant_of_sink_and_dummy(fill):
         p.check_cache()
         p.check_attention(dense=False, step=i)
     p.check_attention(dense=True)
-    L = w.block_tokens
-    assert abs(p.hc.attend_flops(False) - orc.attend_flops(p.geom, w.labels, 4, w.head_dim)
-               - 2 * 4.0 * L * L * w.head_dim) < 1.0  # the 2 Sink/Dummy heads read one more block each
+    assert abs(p.hc.attend_flops(False) - orc.attend_flops(p.geom, w.labels, 4, w.head_dim, sd_blocks=2)) < 1.0
 
 
 def test_refresh_of_the_current_block_in_one_block_mode():

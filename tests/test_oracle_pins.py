@@ -290,6 +290,63 @@ def test_scores_follow_their_definitions_on_a_hand_case():
     assert labels[0] == orc.SPATIAL
 
 
+def _hand_case(v_blocks, r=0, gamma=2.0):
+    """1 x 3 grid, one frame per block, one head, d = 2, every key zero (uniform weights over a key set)."""
+    geom = orc.Geometry.make(1, 3, 1, 10, 10)
+    cache = orc.CacheModel(len(v_blocks), 1)
+    zero = np.zeros((3, 1, 2), np.uint16)
+    for vb in v_blocks:
+        cache.append(zero, synth.f32_to_bf16_bits(np.asarray(vb, np.float32).reshape(3, 1, 2)))
+    q = synth.f32_to_bf16_bits(np.ones((3, 1, 2), np.float32))
+    return orc.classify(q, cache, geom, r=r, gamma=gamma)
+
+
+def test_masked_proxy_and_error_term_on_a_hand_case_with_nonzero_error():
+    # three cached frames (first / middle / newest block); with r = 0 the proxy of the query at column x sees the
+    # three keys of column x only.  Weights are uniform, so every output is a plain average of value rows:
+    #   O_ref  = (4.5, 4.5) / 9 = (1/2, 1/2) for every query
+    #   O_sp   = (2.5, 0.5)/3, (1.25, 1.5)/3, (0.75, 2.5)/3   (column sums of the three blocks)
+    #   O_sink = (2.75, 0.75)/3, O_dummy = (0.25, 2.25)/3
+    v_first = [(2, 0), (0.5, 0.25), (0.25, 0.5)]
+    v_mid = [(0.5, 0.5)] * 3
+    v_last = [(0, 0), (0.25, 0.75), (0, 1.5)]
+    labels, s = _hand_case([v_first, v_mid, v_last], r=0, gamma=2.0)
+    r2 = math.sqrt(2.0)
+    # the cosine with a vector along (1, 1) is (a0 + a1) / (sqrt(2) |a|)
+    cos_sp = [3.0 / (r2 * math.sqrt(6.5)), 2.75 / (r2 * math.sqrt(3.8125)), 3.25 / (r2 * math.sqrt(6.8125))]
+    cos_sink = 3.5 / (r2 * math.sqrt(2.75 ** 2 + 0.75 ** 2))
+    cos_dummy = 2.5 / (r2 * math.sqrt(0.25 ** 2 + 2.25 ** 2))
+    lo, mid = sorted(cos_sp)[:2]
+    p5 = lo + 0.1 * (mid - lo)  # rank 0.05 * (3 - 1)
+    # squared errors per query: |O_sp - (1/2, 1/2)|^2, averaged over L * d = 6 elements
+    sq = [(2.5 / 3 - 0.5) ** 2 + (0.5 / 3 - 0.5) ** 2, (1.25 / 3 - 0.5) ** 2 + 0.0, (0.25 - 0.5) ** 2 + (2.5 / 3 - 0.5) ** 2]
+    mse = sum(sq) / 6.0
+    assert abs(mse - (1 / 9 + 1 / 9 + 1 / 144 + 1 / 16 + 1 / 9) / 6) < 1e-15 and mse > 0.06
+    want = [cos_sink, cos_dummy, sum(cos_sp) / 3, p5, mse, p5 - 2.0 * mse, 1 / 3, 1 / 3, 1 / 3, 2 / 9]
+    assert np.abs(s[0] - np.array(want)).max() < 1e-12
+    assert labels[0] == orc.GLOBAL
+    # gamma enters once, with a minus sign, and multiplies the error only
+    _, s5 = _hand_case([v_first, v_mid, v_last], r=0, gamma=5.0)
+    assert abs(s5[0, 5] - (p5 - 5.0 * mse)) < 1e-12 and abs(s5[0, 3] - p5) < 1e-12
+    # r = 1: the middle column sees the whole frame (error 0 there), the outer columns two of three columns
+    _, s1 = _hand_case([v_first, v_mid, v_last], r=1, gamma=2.0)
+    o_left = np.array([2.5 + 1.25, 0.5 + 1.5]) / 6
+    o_right = np.array([1.25 + 0.75, 1.5 + 2.5]) / 6
+    mse1 = (((o_left - 0.5) ** 2).sum() + ((o_right - 0.5) ** 2).sum()) / 6.0
+    assert abs(s1[0, 4] - mse1) < 1e-15 and abs(s1[0, 8] - (6 + 9 + 6) / 27) < 1e-15 and abs(s1[0, 9] - 2 / 27) < 1e-15
+
+
+def test_zero_norm_output_gives_cosine_zero():
+    # the proxy output of column 0 is exactly the zero vector: its cosine is 0 (clamped denominator), not NaN
+    v_first = [(1, 0), (0.5, 0.25), (0.25, 0.5)]
+    v_last = [(-1, 0), (0.25, 0.75), (0, 1.5)]
+    labels, s = _hand_case([v_first, v_last], r=0)
+    assert np.isfinite(s).all()
+    o_ref = np.array([1.0, 3.0]) / 6
+    cos = [0.0] + [float(a @ o_ref / np.linalg.norm(a) / np.linalg.norm(o_ref)) for a in (np.array([0.75, 1.0]), np.array([0.25, 2.0]))]
+    assert abs(s[0, 2] - sum(cos) / 3) < 1e-12 and abs(s[0, 3] - 0.1 * min(cos[1:])) < 1e-12
+
+
 def test_total_probability_identity_and_mass_partition():
     w = synth.small(n_blocks=3)
     geom, cache = fill(w)
@@ -378,6 +435,10 @@ def test_attend_flops_counts():
     dense = 12 * 4.0 * L * 7 * L * 128
     assert abs(dense / 1e9 - 942.0) < 0.5
     assert abs(orc.attend_flops(geom, labels, 7, 128) / 1e9 - 312.5) < 0.5
+    # the appendix's accounting: Sink / Dummy read two blocks, i.e. one more L x L product per such head
+    two = orc.attend_flops(geom, labels, 7, 128, sd_blocks=2)
+    assert two - orc.attend_flops(geom, labels, 7, 128) == 5 * 4.0 * L * L * 128
+    assert orc.attend_flops(geom, labels, 1, 128, sd_blocks=2) == orc.attend_flops(geom, labels, 1, 128)
 
 
 # ---- the input generator -----------------------------------------------------------------
