@@ -63,6 +63,13 @@ enum {
   HC_N_SCORES = 10
 };
 
+/* Decision rule of headcast_classify. */
+enum {
+  HC_RULE_COSINE = 0, /* Eq. 5 of the paper: mean cosines and the Spatial score against their thresholds */
+  HC_RULE_MASS = 1    /* not in the paper: the same cascade on the mean attention masses (first block, newest block,
+                         (2r+1)^2 neighbourhood) against one threshold mass_tau */
+};
+
 typedef struct headcast_config {
   int32_t n_heads;          /* H, 1..64 */
   int32_t head_dim;         /* d, 64 or 128 */
@@ -86,6 +93,9 @@ typedef struct headcast_config {
   int32_t sd_mode;          /* 0: Sink and Dummy heads keep exactly one block (Sec. 4.3, 4.4).  1: the accounting of
                                Appendix B / C: Sink keeps its anchor block plus the current block, Dummy the previous
                                plus the current block (2L tokens each) */
+  int32_t rule;             /* HC_RULE_COSINE (default, Eq. 5) or HC_RULE_MASS */
+  float mass_tau;           /* HC_RULE_MASS only: Sink if mass_first >= tau, else Dummy if mass_last >= tau, else Spatial
+                               if mass_spatial >= tau, else Global.  0 < tau <= 1; default 0.9 (the paper gives none) */
 } headcast_config;
 
 typedef struct headcast_ctx headcast_ctx;
@@ -219,7 +229,7 @@ const char* headcast_last_error(const headcast_ctx* ctx);
  * other allocating routine.  q_dev and out_dev are [n_queries][n_heads][head_dim] bf16, k_dev and v_dev
  * [n_keys][n_heads][head_dim] bf16, all caller-owned, 16-byte aligned and contiguous.
  *
- * The scratch the kernel needs (work list, tensor maps, status word; about 140 KB) is a fixed device array inside
+ * The scratch the kernel needs in global memory (work list, per-CTA ranges, status word; about 140 KB) is a fixed device array inside
  * the library: every GPU that loads the library holds it until the process exits.  Consequences:
  *   - size limit: n_heads * ceil(n_queries / 256) <= HEADCAST_NOALLOC_MAX_ITEMS, head_dim 64 or 128,
  *     n_heads <= 64; anything larger returns HC_ERR_UNSUPPORTED and does nothing;
@@ -227,7 +237,9 @@ const char* headcast_last_error(const headcast_ctx* ctx);
  *     it uses and clears the status word): two calls whose GPU work overlaps - different streams, or different
  *     host threads - race on it.  Keep calls on one GPU in one stream, or order them with events;
  *   - the first call on each device looks up the array's device address and sets the kernel's shared-memory
- *     attribute (with that device current).  Make that first call before starting any stream capture.
+ *     attribute (with that device current).  Make that first call before starting any stream capture;
+ *   - a call on a stream that is being captured returns HC_ERR_UNSUPPORTED (the work list is copied from a host
+ *     image that the next call rewrites).
  * softmax_scale = 0 selects 1/sqrt(head_dim).  Asynchronous on `stream`.  headcast_noalloc_status synchronises
  * the stream and reports HC_ERR_TIMEOUT if the kernel gave up on a bounded wait; headcast_noalloc_last_error
  * returns the reason of the last failing call (process-wide buffer). */

@@ -30,7 +30,7 @@ MSE = mean over all L*d elements; cosine denominator clamped at 1e-12.
 
 Parity unpinned (the paper prints no worked example): the percentile
 interpolation rule, the cell rounding rule, and the attention-mass auxiliary
-outputs' "rest" partition.  Everything else is pinned by the CPU test suite.
+outputs' "rest" partition, and the threshold of the optional mass rule (``decide_mass``).  Everything else is pinned by the CPU test suite.
 """
 from __future__ import annotations
 
@@ -288,6 +288,18 @@ def decide(cos_sink: float, cos_dummy: float, cos_spatial: float, score: float,
     return GLOBAL
 
 
+def decide_mass(mass_first: float, mass_last: float, mass_spatial: float, tau: float = 0.9) -> int:
+    """The cascade of Eq. 5 applied to the mean attention masses instead of the cosines (not in the paper, which
+    gives no threshold for it: parity unpinned beyond the truth table): same order, same >=, NaN fails every test."""
+    if mass_first >= tau:
+        return SINK
+    if mass_last >= tau:
+        return DUMMY
+    if mass_spatial >= tau:
+        return SPATIAL
+    return GLOBAL
+
+
 def _row_cosine(a: np.ndarray, b: np.ndarray) -> np.ndarray:
     num = (a * b).sum(axis=1)
     den = np.maximum(np.linalg.norm(a, axis=1) * np.linalg.norm(b, axis=1), 1e-12)
@@ -305,7 +317,8 @@ def proxy_allowed(geom: Geometry, rows: np.ndarray, n_keys: int, r: int) -> np.n
 def classify(q_bits: np.ndarray, cache: CacheModel, geom: Geometry, r: int = 2, gamma: float = 5.0,
              thetas: Tuple[float, float, float, float] = (0.95, 0.95, 0.95, 0.755),
              softmax_scale: float = 0.0, rows: Optional[np.ndarray] = None,
-             heads: Optional[Sequence[int]] = None, chunk: int = 256, want_tokens: bool = False):
+             heads: Optional[Sequence[int]] = None, chunk: int = 256, want_tokens: bool = False,
+             rule: int = 0, mass_tau: float = 0.9):
     """One-time head classification (Sec. 4.2).  Returns (labels [H] int32, scores [H, N_SCORES]).
     With ``rows`` given, the per-token quantities are only formed for those rows (the per-head
     statistics are then statistics of that sample).  ``want_tokens`` also returns the per-token
@@ -346,8 +359,12 @@ def classify(q_bits: np.ndarray, cache: CacheModel, geom: Geometry, r: int = 2, 
         p5 = percentile_linear(cos[2], 5.0)
         mse = sqerr.sum() / (rows.size * d)
         score = p5 - gamma * mse  # Eq. 4
-        labels[h] = decide(cs, cd, csp, score, *thetas)  # Eq. 5
-        scores[h] = (cs, cd, csp, p5, mse, score, *mass.mean(axis=1))
+        mean_mass = mass.mean(axis=1)
+        if rule == 0:
+            labels[h] = decide(cs, cd, csp, score, *thetas)  # Eq. 5
+        else:
+            labels[h] = decide_mass(mean_mass[0], mean_mass[1], mean_mass[2], mass_tau)
+        scores[h] = (cs, cd, csp, p5, mse, score, *mean_mass)
         if want_tokens:
             tokens[h] = dict(cos=cos, sqerr=sqerr, mass=mass)
     return (labels, scores, tokens) if want_tokens else (labels, scores)

@@ -34,7 +34,10 @@ class Config(C.Structure):
                 ("col_edges_host", C.POINTER(C.c_int32)), ("n_col_edges", C.c_int32),
                 ("proxy_radius", C.c_int32), ("theta_sink", C.c_float), ("theta_dummy", C.c_float),
                 ("theta_spatial", C.c_float), ("theta_score", C.c_float), ("gamma", C.c_float),
-                ("softmax_scale", C.c_float), ("keep_monolithic", C.c_int32), ("sd_mode", C.c_int32)]
+                ("softmax_scale", C.c_float), ("keep_monolithic", C.c_int32), ("sd_mode", C.c_int32),
+                ("rule", C.c_int32), ("mass_tau", C.c_float)]
+
+RULE_COSINE, RULE_MASS = 0, 1
 
 
 class HeadCastError(RuntimeError):
@@ -104,13 +107,40 @@ def _stream() -> int:
     return torch.cuda.current_stream().cuda_stream
 
 
-def _ptr(t) -> int:
-    assert t.is_cuda and t.is_contiguous(), "tensors handed to the library must be contiguous CUDA tensors"
+def _validate(t, name: str, shape, cuda: bool = True) -> None:
+    """Rejects, before the library sees a pointer, any tensor that would make a kernel read or write outside the
+    caller's buffer: wrong dtype, rank, shape, device or a non-contiguous view.  ``shape`` entries of None are free."""
+    import torch
+    if not isinstance(t, torch.Tensor):
+        raise ValueError(f"{name}: expected a torch tensor, got {type(t).__name__}")
+    if t.dtype != torch.bfloat16:
+        raise ValueError(f"{name}: dtype must be bfloat16, got {t.dtype}")
+    if t.dim() != len(shape) or any(want is not None and int(got) != int(want) for got, want in zip(t.shape, shape)):
+        raise ValueError(f"{name}: shape must be {tuple(shape)}, got {tuple(t.shape)}")
+    if not t.is_contiguous():
+        raise ValueError(f"{name}: must be contiguous")
+    if cuda:
+        if not t.is_cuda:
+            raise ValueError(f"{name}: must be a CUDA tensor")
+        if t.device.index != torch.cuda.current_device():
+            raise ValueError(f"{name}: lives on cuda:{t.device.index}, the current device is cuda:{torch.cuda.current_device()}")
+    elif t.is_cuda:
+        raise ValueError(f"{name}: the host entry points take CPU tensors")
+
+
+def _ptr(t, name: str = "tensor", shape=None) -> int:
+    if shape is not None:
+        _validate(t, name, shape)
+    elif not (t.is_cuda and t.is_contiguous()):
+        raise ValueError(f"{name}: tensors handed to the library must be contiguous CUDA tensors")
     return t.data_ptr()
 
 
-def _host_ptr(t) -> int:
-    assert (not t.is_cuda) and t.is_contiguous(), "host entry points take contiguous CPU tensors"
+def _host_ptr(t, name: str = "tensor", shape=None) -> int:
+    if shape is not None:
+        _validate(t, name, shape, cuda=False)
+    elif t.is_cuda or not t.is_contiguous():
+        raise ValueError(f"{name}: host entry points take contiguous CPU tensors")
     return t.data_ptr()
 
 
@@ -144,9 +174,12 @@ def dense_attend_noalloc(q, k, v, out, softmax_scale: float = 0.0) -> None:
     one GPU share a fixed scratch array inside the library: keep them on one stream.  Sizes beyond
     n_heads * ceil(Lq / 256) <= 2048 are rejected."""
     lib = load_library()
+    if getattr(q, "ndim", 0) != 3 or getattr(k, "ndim", 0) != 3:
+        raise ValueError("q and k must be [rows, heads, head_dim]")
     n_q, h, d = q.shape
-    rc = lib.headcast_dense_attend_noalloc(_ptr(q), _ptr(k), _ptr(v), _ptr(out), n_q, k.shape[0], h, d,
-                                           float(softmax_scale), _stream())
+    n_k = k.shape[0]
+    rc = lib.headcast_dense_attend_noalloc(_ptr(q, "q", (n_q, h, d)), _ptr(k, "k", (n_k, h, d)), _ptr(v, "v", (n_k, h, d)),
+                                           _ptr(out, "out", (n_q, h, d)), n_q, n_k, h, d, float(softmax_scale), _stream())
     if rc != 0:
         raise HeadCastError(rc, lib.headcast_noalloc_last_error().decode())
 
@@ -192,6 +225,10 @@ class HeadCast:
     def from_workload(cls, w, **kw) -> "HeadCast":
         return cls(w.n_heads, w.head_dim, w.grid_h, w.grid_w, w.n_blocks, w.frames_per_block, w.cell_h, w.cell_w, **kw)
 
+    @property
+    def _block(self):
+        return (self.block_tokens, self.n_heads, self.head_dim)
+
     def _check(self, rc: int) -> None:
         if rc != 0:
             raise HeadCastError(rc, self.lib.headcast_last_error(self._ctx).decode())
@@ -208,23 +245,25 @@ class HeadCast:
             pass
 
     def append(self, k_new, v_new) -> None:
-        self._check(self.lib.headcast_append(self._ctx, _ptr(k_new), _ptr(v_new), _stream()))
+        self._check(self.lib.headcast_append(self._ctx, _ptr(k_new, "k_new", self._block), _ptr(v_new, "v_new", self._block), _stream()))
 
     def overwrite_last(self, k_new, v_new) -> None:
-        self._check(self.lib.headcast_overwrite_last(self._ctx, _ptr(k_new), _ptr(v_new), _stream()))
+        self._check(self.lib.headcast_overwrite_last(self._ctx, _ptr(k_new, "k_new", self._block), _ptr(v_new, "v_new", self._block), _stream()))
 
     def full_attend(self, q, out) -> None:
-        self._check(self.lib.headcast_full_attend(self._ctx, _ptr(q), _ptr(out), _stream()))
+        self._check(self.lib.headcast_full_attend(self._ctx, _ptr(q, "q", self._block), _ptr(out, "out", self._block), _stream()))
 
     def classify(self, q):
         import numpy as np
         labels = (C.c_int32 * self.n_heads)()
         scores = (C.c_float * (self.n_heads * N_SCORES))()
-        self._check(self.lib.headcast_classify(self._ctx, _ptr(q), labels, scores, _stream()))
+        self._check(self.lib.headcast_classify(self._ctx, _ptr(q, "q", self._block), labels, scores, _stream()))
         return (np.array(labels[:], dtype=np.int32),
                 np.array(scores[:], dtype=np.float32).reshape(self.n_heads, N_SCORES))
 
     def set_labels(self, labels: Sequence[int]) -> None:
+        if len(labels) != self.n_heads:
+            raise ValueError(f"labels: expected {self.n_heads} entries, got {len(labels)}")
         arr = (C.c_int32 * self.n_heads)(*[int(v) for v in labels])
         self._check(self.lib.headcast_set_labels(self._ctx, arr))
 
@@ -237,15 +276,15 @@ class HeadCast:
         self._check(self.lib.headcast_split_cache(self._ctx, _stream()))
 
     def attend(self, q, out) -> None:
-        self._check(self.lib.headcast_attend(self._ctx, _ptr(q), _ptr(out), _stream()))
+        self._check(self.lib.headcast_attend(self._ctx, _ptr(q, "q", self._block), _ptr(out, "out", self._block), _stream()))
 
     def append_host(self, k_host, v_host) -> None:
         """k_host / v_host: CPU tensors (pinned for overlap) of shape [L, H, d], bf16."""
-        self._check(self.lib.headcast_append_host(self._ctx, _host_ptr(k_host), _host_ptr(v_host), _stream()))
+        self._check(self.lib.headcast_append_host(self._ctx, _host_ptr(k_host, "k_host", self._block), _host_ptr(v_host, "v_host", self._block), _stream()))
 
     def attend_host(self, q_host, out_host) -> None:
         """q_host / out_host: CPU tensors (pinned for overlap); out_host is complete after the stream is synchronised."""
-        self._check(self.lib.headcast_attend_host(self._ctx, _host_ptr(q_host), _host_ptr(out_host), _stream()))
+        self._check(self.lib.headcast_attend_host(self._ctx, _host_ptr(q_host, "q_host", self._block), _host_ptr(out_host, "out_host", self._block), _stream()))
 
     def export_cache_device(self, head: int):
         """Returns (K, V) bf16 device tensors [n_tokens, d] of what the cache keeps for ``head``, logical order."""

@@ -22,17 +22,6 @@
 
 namespace hc {
 
-// Development aid, compiled out unless HC_TIMELINE is defined: CTA 0 stamps the global timer at the hand-over
-// points of its first 64 key tiles into AttnParams::trace, behind the per-item area (16 slots per tile).
-#ifdef HC_TIMELINE
-#define HC_STAMP(iter, slot)                                                                      \
-  do {                                                                                            \
-    if (p.trace && blockIdx.x == 0 && (iter) < 64) p.trace[p.trace_base + (iter) * 16 + (slot)] = global_timer_ns(); \
-  } while (0)
-#else
-#define HC_STAMP(iter, slot) do { } while (0)
-#endif
-
 struct CellGeom {
   int32_t y0, x0, ch, cw;  // top-left grid position and extent of a deployed Spatial cell
 };
@@ -59,7 +48,6 @@ struct WorkItem {
 struct AttnParams {
   const WorkItem* items;
   const int32_t* cta_first;  // [gridDim.x + 1]: CTA b owns items [cta_first[b], cta_first[b + 1])
-  const CUtensorMap* maps;
   const CellGeom* cells;
   const __nv_bfloat16* q;  // [L][H][d]
   __nv_bfloat16* out;      // [L][H][d]
@@ -71,11 +59,14 @@ struct AttnParams {
   int32_t n_heads, tokens_per_frame, grid_w, block_tokens;
   float scale_log2e;       // softmax scale * log2(e)
   int32_t* status;
-  int32_t trace_base;         // HC_TIMELINE only: first timeline slot inside `trace`
   unsigned long long* trace;  // optional [2 * n_items]: globaltimer (ns) when query tile 0's warpgroup starts / ends an item
   // Spatial proxy only
   int32_t radius;
   int32_t mid_seg_lo, mid_seg_hi, last_seg_lo, last_seg_hi;  // segments (cached frames) of the middle / newest blocks
+  // K map = maps[2 * kv_map], V map = maps[2 * kv_map + 1].  The descriptors travel in the kernel's parameter space
+  // (the kernel takes its parameters as __grid_constant__), so a launch always reads the descriptors it was given:
+  // no copy to global memory, nothing another launch can overwrite, no tensor-map proxy fence to forget.
+  alignas(64) CUtensorMap maps[8];
 };
 
 constexpr int ATTN_THREADS = 576;  // warp 0: TMA, warp 1: MMA, warps 2-9 / 10-17: softmax for query tile 0 / 1 (112 registers each)
@@ -144,7 +135,7 @@ __device__ __forceinline__ void apply_visible(uint32_t (&sv)[32], uint32_t visib
 }
 
 template <int D, bool PROXY>
-__global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const AttnParams p) {
+__global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const __grid_constant__ AttnParams p) {
   using SM = AttnSmem<D>;
   constexpr int NB = D / 64;          // 64-column blocks per tile
   constexpr int QK_STEPS = D / 16;    // k-steps of S = Q K^T
@@ -272,19 +263,15 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const AttnParams 
           const uint32_t st = gv % KV_SLOTS, ph = (gv / KV_SLOTS) & 1;
           const uint32_t st1 = gk % KV_SLOTS, ph1 = (gk / KV_SLOTS) & 1;
           if (!(ok = mbar_wait(&bar_kv_full[st], ph, abortp, p.status, 23))) break;
-          HC_STAMP(kt + j, 0);
           for (int t = 0; t < n_q && ok; ++t) {
             if (!(ok = mbar_wait(&bar_p_full[t], p_cnt[t] & 1, abortp, p.status, 24))) break;
-            HC_STAMP(kt + j, 1 + 3 * t);
             ++p_cnt[t];
             tc_fence_after_sync();
             issue_pv(t, st, j > 0);
-            HC_STAMP(kt + j, 2 + 3 * t);
             if (j + 1 < nt) {
               if (t == 0 && !(ok = mbar_wait(&bar_kv_full[st1], ph1, abortp, p.status, 25))) break;
               tc_fence_after_sync();
               issue_qk(t, st1);
-              HC_STAMP(kt + j, 3 + 3 * t);
               mma_commit(&bar_s_full[t]);
               if (t == n_q - 1) mma_commit(&bar_kv_free[st1]);
             } else {
@@ -364,7 +351,6 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const AttnParams 
         const int n_valid = min(128, w.seg_len - c * 128) - half * 64;  // valid keys among this thread's 64
         const int tok0 = PROXY ? (w.kv_row0 + c * 128 + half * 64) : 0;  // in-frame token of its first key
         if (!(ok = mbar_wait(&bar_s_full[t], s_cnt & 1, abortp, p.status, 31))) break;
-        if (r == 0 && half == 0) HC_STAMP(s_cnt, 7 + 4 * t);
         ++s_cnt;
         tc_fence_after_sync();
         // pass 1: maximum of this thread's 64 logits (32 columns at a time; they are read again in pass 2, which
@@ -391,11 +377,9 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const AttnParams 
           }
           mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
         }
-        if (r == 0 && half == 0) HC_STAMP(s_cnt - 1, 8 + 4 * t);
         float mx_other;
         if (!(ok = swap_with_partner(mx, mx_other))) break;
         mx = fmaxf(mx, mx_other) * p.scale_log2e;  // row maximum; scale > 0, so the maximum commutes with it
-        if (r == 0 && half == 0) HC_STAMP(s_cnt - 1, 9 + 4 * t);
         // running maximum: move the reference only when some row of the warp outgrew it by 2^8.  Both threads of
         // a row see the same maximum and sit in the same lane of their warps, so both warps decide alike.
         const bool grow = mx > m_ref + RESCALE_THRESHOLD || (m_ref == -INFINITY && mx > -INFINITY);
@@ -464,7 +448,6 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const AttnParams 
         tc_fence_before_sync();
         __syncwarp();
         if (lane == 0) mbar_arrive(&bar_p_full[t]);
-        if (r == 0 && half == 0) HC_STAMP(s_cnt - 1, 10 + 4 * t);
       }
       if (!ok) break;
       // ---- epilogue: row sums of the two halves are added, each thread normalises and stores its output columns

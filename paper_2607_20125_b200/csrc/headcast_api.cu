@@ -93,7 +93,7 @@ struct headcast_ctx {
   __nv_bfloat16 *sd_k = nullptr, *sd_v = nullptr, *g_k = nullptr, *g_v = nullptr, *sp_k = nullptr, *sp_v = nullptr;
   int32_t *sp_base = nullptr, *sp_nc = nullptr;
   CellGeom* cells_dev = nullptr;
-  CUtensorMap* maps_dev = nullptr;
+  CUtensorMap maps[2 * N_MAP_PAIRS];  // host copies; every attention launch carries them as kernel parameters
   int32_t* status_dev = nullptr;
 
   Schedule sched_dense, sched_hc, sched_cls, sched_proxy;
@@ -166,8 +166,8 @@ size_t cache_elems(const headcast_ctx* c, int heads) {
 
 // ---------------------------------------------------------------------------------- tensor maps
 int build_maps(headcast_ctx* c) {
-  CUtensorMap maps[2 * N_MAP_PAIRS];
-  std::memset(maps, 0, sizeof(maps));
+  CUtensorMap* maps = c->maps;
+  std::memset(maps, 0, sizeof(c->maps));
   const uint64_t win_rows = static_cast<uint64_t>(c->n_blk) * c->L;
   bool ok = true;
   if (c->mono_k) {
@@ -192,7 +192,6 @@ int build_maps(headcast_ctx* c) {
     ok = ok && make_tmap_bf16_2d(&maps[2 * MAP_SPATIAL + 1], c->sp_v, c->D, rows, c->D, 128);
   }
   if (!ok) return fail(c, HC_ERR_CUDA, "cuTensorMapEncodeTiled failed or is unavailable");
-  HC_CUDA(c, cudaMemcpy(c->maps_dev, maps, sizeof(maps), cudaMemcpyHostToDevice));
   return HC_OK;
 }
 
@@ -577,6 +576,10 @@ int upload_schedule(headcast_ctx* c, Schedule& s, cudaStream_t st) {
     HC_CUDA(c, c->part_ml.reserve(static_cast<size_t>(s.n_slots) * 256));
     HC_CUDA(c, c->part_mid.reserve(static_cast<size_t>(s.n_slots) * 256));
   }
+  // The lists are uploaded once per cache fill and reused by later calls, which may come on another stream: wait
+  // here, once, so that no later launch can see a half-written list (the host vectors are pageable, so the copies
+  // have mostly completed by now anyway).
+  HC_CUDA(c, cudaStreamSynchronize(st));
   s.uploaded = true;
   return HC_OK;
 }
@@ -612,7 +615,8 @@ int run_schedule(headcast_ctx* c, Schedule& s, const void* q, void* out, bool pr
   std::memset(&p, 0, sizeof(p));
   p.items = s.items_dev.ptr;
   p.cta_first = s.cta_first_dev.ptr;
-  p.maps = c->maps_dev;
+  static_assert(sizeof(p.maps) == sizeof(c->maps), "one K and one V map per buffer");
+  std::memcpy(p.maps, c->maps, sizeof(p.maps));
   p.cells = c->cells_dev;
   p.q = static_cast<const __nv_bfloat16*>(q);
   p.out = static_cast<__nv_bfloat16*>(out);
@@ -629,11 +633,10 @@ int run_schedule(headcast_ctx* c, Schedule& s, const void* q, void* out, bool pr
   p.status = c->status_dev;
   p.trace = nullptr;
   if (c->tracing) {
-    const size_t trace_words = 2 * s.items.size() + 16 * 64;  // per-item stamps, then the HC_TIMELINE area
+    const size_t trace_words = 2 * s.items.size();
     HC_CUDA(c, c->trace_dev.reserve(trace_words));
     HC_CUDA(c, cudaMemsetAsync(c->trace_dev.ptr, 0, trace_words * sizeof(unsigned long long), st));
     p.trace = c->trace_dev.ptr;
-    p.trace_base = static_cast<int32_t>(2 * s.items.size());
     c->trace_items = s.items;
     c->trace_cta_first = s.cta_first;
   }
@@ -785,7 +788,8 @@ static int init_host(headcast_ctx* c, const headcast_config* cfg, std::vector<in
   if (cfg->n_heads < 1 || cfg->n_heads > MAX_HEADS || (cfg->head_dim != 64 && cfg->head_dim != 128) ||
       cfg->grid_h < 1 || cfg->grid_w < 1 || cfg->frames_per_block < 1 || cfg->n_blocks < 2 ||
       cfg->n_blocks > MAX_BLOCKS || cfg->cell_h < 1 || cfg->cell_w < 1 || cfg->proxy_radius < 0 ||
-      !(cfg->softmax_scale >= 0.0f) || cfg->sd_mode < 0 || cfg->sd_mode > 1)
+      !(cfg->softmax_scale >= 0.0f) || cfg->sd_mode < 0 || cfg->sd_mode > 1 || cfg->rule < 0 || cfg->rule > 1 ||
+      (cfg->rule == 1 && !(cfg->mass_tau > 0.0f && cfg->mass_tau <= 1.0f)))
     return HC_ERR_INVALID_ARG;
   const long long L = static_cast<long long>(cfg->frames_per_block) * cfg->grid_h * cfg->grid_w;
   if (L * cfg->n_blocks * cfg->n_heads * cfg->head_dim >= (1LL << 40) || L * cfg->n_blocks * cfg->n_heads >= (1LL << 31))
@@ -850,6 +854,8 @@ void headcast_default_config(headcast_config* cfg) {
   cfg->theta_score = 0.755f;
   cfg->gamma = 5.0f;
   cfg->softmax_scale = 0.0f;
+  cfg->rule = HC_RULE_COSINE;
+  cfg->mass_tau = 0.9f;
 }
 
 int headcast_create(const headcast_config* cfg, headcast_ctx** out) {
@@ -886,7 +892,6 @@ int headcast_create(const headcast_config* cfg, headcast_ctx** out) {
   step(cudaMalloc(&c->sp_base, c->T_f * sizeof(int32_t)));
   step(cudaMalloc(&c->sp_nc, c->T_f * sizeof(int32_t)));
   step(cudaMalloc(&c->cells_dev, c->cells.size() * sizeof(CellGeom)));
-  step(cudaMalloc(&c->maps_dev, 2 * N_MAP_PAIRS * sizeof(CUtensorMap)));
   step(cudaMalloc(&c->status_dev, sizeof(int32_t)));
   if (e == cudaSuccess) {
     step(cudaMemset(c->mono_k, 0, mono_bytes));
@@ -913,7 +918,7 @@ int headcast_create(const headcast_config* cfg, headcast_ctx** out) {
 int headcast_destroy(headcast_ctx* c) {
   if (!c) return HC_OK;
   cudaDeviceSynchronize();
-  void* ptrs[] = {c->mono_k, c->mono_v, c->arena_k, c->arena_v, c->sp_base, c->sp_nc, c->cells_dev, c->maps_dev, c->status_dev};
+  void* ptrs[] = {c->mono_k, c->mono_v, c->arena_k, c->arena_v, c->sp_base, c->sp_nc, c->cells_dev, c->status_dev};
   for (void* p : ptrs)
     if (p) cudaFree(p);
   if (c->ev_a) cudaEventDestroy(c->ev_a);
@@ -1158,6 +1163,8 @@ int headcast_classify(headcast_ctx* c, const void* q, int32_t* labels_host, floa
     d.theta_spatial = c->cfg.theta_spatial;
     d.theta_score = c->cfg.theta_score;
     d.gamma = c->cfg.gamma;
+    d.rule = c->cfg.rule;
+    d.mass_tau = c->cfg.mass_tau;
     head_decide_kernel<<<c->H, 512, 0, st>>>(d);
     HC_CUDA(c, cudaGetLastError());
     ++c->launches;
@@ -1446,16 +1453,6 @@ int headcast_read_trace(headcast_ctx* c, int64_t* rows_host, int32_t capacity, i
   return HC_OK;
 }
 
-#ifdef HC_TIMELINE
-int headcast_read_timeline(headcast_ctx* c, int64_t* out_host /* [64][16] */) {
-  if (!c || !out_host || c->trace_items.empty()) return HC_ERR_INVALID_ARG;
-  HC_CUDA(c, cudaDeviceSynchronize());
-  HC_CUDA(c, cudaMemcpy(out_host, c->trace_dev.ptr + 2 * c->trace_items.size(), 16 * 64 * sizeof(int64_t),
-                        cudaMemcpyDeviceToHost));
-  return HC_OK;
-}
-#endif
-
 int headcast_plan_schedule(const headcast_config* cfg, const int32_t* labels_host, int32_t n_filled, int32_t n_ctas,
                            int32_t dense, int32_t* items_host, int32_t capacity, int32_t* n_items_host,
                            int32_t* cta_first_host) {
@@ -1509,8 +1506,9 @@ const char* headcast_last_error(const headcast_ctx* c) { return c ? c->err.c_str
 // =====================================================================================================
 // Allocation-free dense attention
 // =====================================================================================================
-// Everything the attention kernel needs besides the caller's tensors - the work list, the per-CTA ranges, two
-// tensor maps and the status word - lives in one file-scope device array of fixed size.  Each GPU that loads the
+// Everything the attention kernel needs in global memory besides the caller's tensors - the work list, the per-CTA
+// ranges and the status word - lives in one file-scope device array of fixed size (the two tensor maps travel as
+// kernel parameters).  Each GPU that loads the
 // library carries these bytes until the process exits.
 namespace {
 
@@ -1518,7 +1516,6 @@ constexpr int NOALLOC_MAX_ITEMS = HEADCAST_NOALLOC_MAX_ITEMS;
 constexpr int NOALLOC_MAX_CTAS = 1024;
 
 struct NoAllocScratch {
-  CUtensorMap maps[2];                     // K and V of the caller's buffers
   WorkItem items[NOALLOC_MAX_ITEMS];
   int32_t cta_first[NOALLOC_MAX_CTAS + 1];
   int32_t status;
@@ -1590,12 +1587,23 @@ int headcast_dense_attend_noalloc(const void* q, const void* k, const void* v, v
   if (rc != HC_OK) return rc;
   const NoAllocDevice& d = g_noalloc_dev[dev];
   cudaStream_t st = static_cast<cudaStream_t>(stream);
+  {
+    // the work list is copied from a host image that the next call rewrites: a captured copy would re-read it at
+    // every replay, so capturing streams are turned away
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    e = cudaStreamIsCapturing(st, &cap);
+    if (e != cudaSuccess) return noalloc_fail(HC_ERR_CUDA, "cudaStreamIsCapturing", e);
+    if (cap != cudaStreamCaptureStatusNone)
+      return noalloc_fail(HC_ERR_UNSUPPORTED, "headcast_dense_attend_noalloc cannot be called on a capturing stream");
+  }
 
   // host image of the scratch: thread-local static storage, no heap
   static thread_local NoAllocScratch host;
   const uint64_t row_elems = static_cast<uint64_t>(n_heads) * head_dim;
-  if (!make_tmap_bf16_2d(&host.maps[0], k, row_elems, n_keys, row_elems, 128) ||
-      !make_tmap_bf16_2d(&host.maps[1], v, row_elems, n_keys, row_elems, 128))
+  AttnParams p;
+  std::memset(&p, 0, sizeof(p));
+  if (!make_tmap_bf16_2d(&p.maps[0], k, row_elems, n_keys, row_elems, 128) ||
+      !make_tmap_bf16_2d(&p.maps[1], v, row_elems, n_keys, row_elems, 128))
     return noalloc_fail(HC_ERR_CUDA, "cuTensorMapEncodeTiled failed or is unavailable");
   // whole query-tile pairs, dealt round-robin to one CTA per SM (every item has the same key range)
   const int n_cta = d.n_sm;
@@ -1616,19 +1624,14 @@ int headcast_dense_attend_noalloc(const void* q, const void* k, const void* v, v
   }
   host.cta_first[n_cta] = n;
   host.status = 0;  // the array keeps the previous call's contents: the status word must start at zero
-  e = cudaMemcpyAsync(d.scratch->maps, host.maps, sizeof(host.maps), cudaMemcpyHostToDevice, st);
-  if (e == cudaSuccess)
-    e = cudaMemcpyAsync(d.scratch->items, host.items, static_cast<size_t>(n) * sizeof(WorkItem), cudaMemcpyHostToDevice, st);
+  e = cudaMemcpyAsync(d.scratch->items, host.items, static_cast<size_t>(n) * sizeof(WorkItem), cudaMemcpyHostToDevice, st);
   if (e == cudaSuccess)
     e = cudaMemcpyAsync(d.scratch->cta_first, host.cta_first, (n_cta + 1) * sizeof(int32_t), cudaMemcpyHostToDevice, st);
   if (e == cudaSuccess) e = cudaMemcpyAsync(&d.scratch->status, &host.status, sizeof(int32_t), cudaMemcpyHostToDevice, st);
   if (e != cudaSuccess) return noalloc_fail(HC_ERR_CUDA, "copying the work list into the static scratch", e);
 
-  AttnParams p;
-  std::memset(&p, 0, sizeof(p));
   p.items = d.scratch->items;
   p.cta_first = d.scratch->cta_first;
-  p.maps = d.scratch->maps;
   p.q = static_cast<const __nv_bfloat16*>(q);
   p.out = static_cast<__nv_bfloat16*>(out);
   p.n_heads = n_heads;

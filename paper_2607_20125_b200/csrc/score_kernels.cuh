@@ -119,6 +119,8 @@ struct DecideParams {
   int32_t rank_lo;   // floor(0.05 * (L - 1))
   float rank_frac;
   float theta_sink, theta_dummy, theta_spatial, theta_score, gamma;
+  int32_t rule;      // 0: cosine rule of Eq. 5; 1: the same cascade on the mean attention masses
+  float mass_tau;
 };
 
 // One block per head: fixed-order sums (deterministic), percentile by selection, Eq. 4 and Eq. 5.
@@ -164,16 +166,25 @@ __global__ void __launch_bounds__(512) head_decide_kernel(const DecideParams p) 
     const float p5 = lo + p.rank_frac * (hi - lo);
     const float mse = static_cast<float>(sums[TOK_SQERR] / (static_cast<double>(p.L) * p.D));
     const float score = p5 - p.gamma * mse;
+    const float m_first = static_cast<float>(sums[TOK_MASS_FIRST]) * inv_l;
+    const float m_last = static_cast<float>(sums[TOK_MASS_LAST]) * inv_l;
+    const float m_near = static_cast<float>(sums[TOK_MASS_SPATIAL]) * inv_l;
     int label = 3;
-    if (cs >= p.theta_sink) label = 0;
-    else if (cd >= p.theta_dummy) label = 1;
-    else if (csp >= p.theta_spatial && score >= p.theta_score) label = 2;
+    if (p.rule == 1) {  // mass rule: same order of tests, same >=, a NaN fails every comparison
+      if (m_first >= p.mass_tau) label = 0;
+      else if (m_last >= p.mass_tau) label = 1;
+      else if (m_near >= p.mass_tau) label = 2;
+    } else {
+      if (cs >= p.theta_sink) label = 0;
+      else if (cd >= p.theta_dummy) label = 1;
+      else if (csp >= p.theta_spatial && score >= p.theta_score) label = 2;
+    }
     p.labels[h] = label;
     float* s = p.scores + h * 10;
     s[0] = cs; s[1] = cd; s[2] = csp; s[3] = p5; s[4] = mse; s[5] = score;
-    s[6] = static_cast<float>(sums[TOK_MASS_FIRST]) * inv_l;
-    s[7] = static_cast<float>(sums[TOK_MASS_LAST]) * inv_l;
-    s[8] = static_cast<float>(sums[TOK_MASS_SPATIAL]) * inv_l;
+    s[6] = m_first;
+    s[7] = m_last;
+    s[8] = m_near;
     s[9] = static_cast<float>(sums[TOK_MASS_REST]) * inv_l;
   }
 }

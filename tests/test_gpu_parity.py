@@ -195,9 +195,9 @@ def test_wrong_state_calls_change_nothing():
     assert e.value.code == -2
     with pytest.raises(HeadCastError):
         p.hc.set_labels(w.labels)
-    with pytest.raises(HeadCastError) as e:
-        p.hc.attend(q[1:].reshape(-1)[1:], out)  # misaligned pointer
-    assert e.value.code == -1
+    with pytest.raises(ValueError):
+        p.hc.attend(q[1:], out)  # the binding refuses a tensor of the wrong shape
+    assert p.hc.lib.headcast_attend(p.hc._ctx, q.data_ptr() + 2, out.data_ptr(), None) == -1  # misaligned pointer
     p.check_cache()
     assert p.hc.n_filled() == 2
 
@@ -224,6 +224,29 @@ def test_classify_tiny(cell):
     p.cache.split(p.w.labels)
     p.check_cache()
     p.check_attention(dense=False)
+
+
+def test_mass_rule_gives_the_planted_labels_and_follows_its_threshold():
+    # the optional rule on attention masses (same cascade as Eq. 5, one threshold): planted archetypes concentrate their
+    # mass on the first block / newest block / neighbourhood, so it reproduces the labels; labels equal the oracle's
+    w = synth.tiny(cell=4)
+    q = synth.make_q(w, 4, 0)
+    for tau, rule_labels in ((0.9, None), (0.999999, None)):
+        p = Pair(w, rule=1, mass_tau=tau)
+        p.append(5)
+        labels, scores = p.hc.classify(to_dev(q))
+        want_labels, want = orc.classify(q, p.cache, p.geom, rule=1, mass_tau=tau)
+        margin = np.abs(want[:, 6:9] - tau).min()
+        if margin > 1e-2:  # away from the threshold the fp32 masses decide like the float64 ones
+            assert tuple(labels) == tuple(want_labels), (tau, labels, want_labels)
+        assert np.abs(scores[:, 6:].astype(np.float64) - want[:, 6:]).max() <= 5e-3
+        if tau == 0.9:
+            assert tuple(labels) == tuple(w.labels)
+        p.hc.destroy()
+    # the cosine rule is untouched by mass_tau
+    p = Pair(w, rule=0, mass_tau=0.1)
+    p.append(5)
+    assert tuple(p.hc.classify(to_dev(q))[0]) == tuple(w.labels)
 
 
 def test_classify_small_with_ring_rolled_before_classification():

@@ -261,6 +261,25 @@ def test_decision_rule_truth_table():
     assert d(float("nan"), 0.96, 0.3, 0.1) == orc.DUMMY
 
 
+def test_mass_rule_truth_table_and_planted_heads():
+    d = orc.decide_mass
+    assert d(0.9, 0.95, 0.95, 0.9) == orc.SINK  # >= and the first branch wins
+    assert d(0.8999, 0.9, 0.95, 0.9) == orc.DUMMY
+    assert d(0.1, 0.8999, 0.9, 0.9) == orc.SPATIAL
+    assert d(0.1, 0.1, 0.8999, 0.9) == orc.GLOBAL
+    assert d(float("nan"), 0.95, 0.1, 0.9) == orc.DUMMY and d(float("nan"), float("nan"), float("nan"), 0.9) == orc.GLOBAL
+    assert d(0.5, 0.1, 0.1, 0.5) == orc.SINK  # the threshold is the argument, not a constant
+    # planted archetypes concentrate their mass where Appendix A says they do: both rules give the planted labels
+    w = synth.tiny(cell=4)
+    geom, cache = fill(w)
+    q = synth.make_q(w, w.n_blocks - 1, 0)
+    by_cos, s = orc.classify(q, cache, geom)
+    by_mass, s2 = orc.classify(q, cache, geom, rule=1, mass_tau=0.9)
+    assert tuple(by_cos) == tuple(by_mass) == w.labels and np.array_equal(s, s2)
+    # the rule really reads the masses: with a threshold nobody reaches every head is Global
+    assert tuple(orc.classify(q, cache, geom, rule=1, mass_tau=1.0 + 1e-9)[0]) == (orc.GLOBAL,) * 4
+
+
 def test_percentile_rule():
     assert orc.percentile_linear(np.arange(21.0)[::-1], 5.0) == 1.0  # rank 0.05*20 = 1
     assert abs(orc.percentile_linear(np.array([0.0, 10.0, 20.0]), 5.0) - 1.0) < 1e-12  # rank 0.1
