@@ -331,6 +331,86 @@ def test_rollout_sequence_three_layers():
                 p.check_attention(dense=False, rows=rows, step=step)
 
 
+def test_rollout_at_the_720p_grid_two_layers_classified_labels_drive_the_split():
+    # the streaming rollout at its own size (45 x 80 grid, 12 heads x 128, 7-block cache), two layers with different
+    # seeded head mixes: two warm-up blocks with dense attention, the third block appended and classified on the
+    # planted inputs - the labels the GPU returns (equal to the oracle's and to the planted ones) drive the split at 3
+    # cached blocks - then 6 more appends, so the ring fills (7) and rolls twice.  Every block: cache bit-exact for
+    # three exported heads, attention on sampled rows at the first and last denoise step.
+    for layer in (0, 1):
+        w = synth.wan("720p", layer=layer)
+        rows = synth.sample_rows(w, n_random=32)[::7]
+        p = Pair(w, keep_monolithic=(layer == 0))
+        for _ in range(2):
+            p.append()
+            p.check_attention(dense=True, rows=rows)
+        p.append()
+        q = synth.make_q(w, 2, 0)
+        labels, _ = p.hc.classify(to_dev(q))
+        want_labels, _ = orc.classify(q, p.cache, p.geom, rows=rows[::2])
+        assert tuple(int(v) for v in labels) == tuple(int(v) for v in want_labels) == tuple(w.labels)
+        p.hc.split_cache()  # no set_labels: the context splits by what its own classification found
+        p.cache.split([int(v) for v in labels])
+        assert p.hc.n_filled() == 3
+        for block in range(6):
+            p.append()
+            assert p.hc.n_filled() == min(7, 4 + block)
+            for h in [(3 * block + i * 5 + layer) % w.n_heads for i in range(3)]:
+                k, v = p.hc.export_cache(h)
+                ko, vo = p.cache.head_kv_bits(h)
+                assert k.shape == ko.shape and np.array_equal(k, ko) and np.array_equal(v, vo), (layer, block, h)
+            for step in (0, 3):
+                p.check_attention(dense=False, rows=rows, step=step)
+        if layer == 0:
+            p.check_attention(dense=True, rows=rows)  # the monolithic ring kept alongside rolled the same way
+        p.hc.destroy()
+
+
+def test_cuda_graph_replay_of_append_and_attend_matches_eager_bit_for_bit():
+    # the steady state of a rollout captured into CUDA graphs, one per ring position (the slot a new block lands in
+    # cycles with period n_blocks - 1, and after that many appends the host-side ring is back where it started);
+    # replays with fresh data in the static input buffers give the eager context's bytes
+    import torch
+    w = synth.small()
+    eager, graphed = Pair(w, keep_monolithic=False), Pair(w, keep_monolithic=False)
+    for p in (eager, graphed):
+        p.append(w.n_blocks)
+        p.hc.set_labels(w.labels)
+        p.hc.split_cache()
+        p.cache.split(w.labels)
+        p.append()  # the work lists of the full cache are uploaded by this eager step
+        p.check_attention(dense=False, rows=synth.sample_rows(w, n_random=16))
+    L, H, D = w.block_tokens, w.n_heads, w.head_dim
+    k_buf, v_buf, q_buf = (torch.zeros((L, H, D), dtype=torch.bfloat16, device="cuda") for _ in range(3))
+    out_g, out_e = torch.zeros_like(q_buf), torch.zeros_like(q_buf)
+    period = w.n_blocks - 1
+    graphs = []
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        for ph in range(period):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=side):
+                graphed.hc.append(k_buf, v_buf)
+                graphed.hc.attend(q_buf, out_g)
+            graphs.append(g)
+    torch.cuda.synchronize()
+    for i in range(2 * period + 1):
+        k, v = synth.make_kv(w, 50 + i)
+        q = synth.make_q(w, 50 + i, i % 4)
+        k_buf.copy_(to_dev(k)); v_buf.copy_(to_dev(v)); q_buf.copy_(to_dev(q))
+        graphs[i % period].replay()
+        eager.hc.append(to_dev(k), to_dev(v))
+        eager.hc.attend(to_dev(q), out_e)
+        torch.cuda.synchronize()
+        assert torch.equal(out_g, out_e), i
+        graphed.hc.append(k_buf, v_buf)  # keeps the graphed context's host-side ring in step with what the replay did
+        for h in (0, 3):
+            kg, vg = graphed.hc.export_cache(h)
+            ke, ve = eager.hc.export_cache(h)
+            assert np.array_equal(kg, ke) and np.array_equal(vg, ve)
+    eager.hc.check(); graphed.hc.check()
+
+
 def test_an_expired_wait_is_reported_and_the_context_stays_usable():
     # failure detection without a GPU fault: a kernel waits (bounded) on a barrier nothing signals, gives up after
     # 50 ms, the host sees HC_ERR_TIMEOUT, and the same context then computes correct attention
