@@ -473,6 +473,28 @@ def measure_copy_path(w, kv, torch, HeadCast, flush, sd_mode):
     b.synchronize()
     res["append_back_to_back_ms"] = a.elapsed_time(b) / n_b2b
     res["append_back_to_back_gbs"] = nbytes["append"] / res["append_back_to_back_ms"] / 1e6
+    # the same 200 appends as ONE CUDA graph launch: no host work between the kernels (the eager loop above pays a
+    # Python call per 10-50 us kernel).  Capture records the launches and advances the host-side ring exactly as the
+    # replay then advances the device-side one.
+    try:
+        graph = torch.cuda.CUDAGraph()
+        side = torch.cuda.Stream()
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(graph, stream=side):
+                for i in range(n_b2b):
+                    hc.append(*kv[w.n_blocks + i % n_extra])
+        torch.cuda.synchronize()
+        flush()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        graph.replay()
+        b.record()
+        b.synchronize()
+        res["append_graph_ms"] = a.elapsed_time(b) / n_b2b
+        res["append_graph_gbs"] = nbytes["append"] / res["append_graph_ms"] / 1e6
+    except Exception as exc:  # report, do not hide
+        res["append_graph_ms"] = None
+        res["append_graph_error"] = str(exc)[:200]
     hc.check()
     hc.destroy()
     return res
@@ -751,6 +773,9 @@ def main():
                     help="heads: one layer's heads spread over the ranks (strong scaling) instead of one replica per GPU")
     ap.add_argument("--pathways", default=None, metavar="FILE",
                     help="also write a per-pathway table (share of FLOPs vs share of CTA time, from the per-item trace) to FILE")
+    ap.add_argument("--copy-only", action="store_true",
+                    help="only the method's byte movement of one workload (split and appends without a monolithic cache): "
+                         "a short run for profiler captures of the copy kernel")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-phases", action="store_true")
     args = ap.parse_args()
@@ -778,6 +803,13 @@ def main():
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     peaks = measured_peaks()
+    if args.copy_only:
+        w = workload_of(headline)
+        flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+        kv, _, _ = gen_inputs(w, 2, torch)
+        res = measure_copy_path(w, kv, torch, HeadCast, lambda: flush_buf.zero_(), args.sd_mode)
+        print(json.dumps({"workload": w.name, "copy_path_method_only": res, "hbm_peak_gbs": peaks["hbm_gbs"]}))
+        return
 
     per = {}
     for name in names:

@@ -141,8 +141,8 @@ int headcast_get_labels(const headcast_ctx* ctx, int32_t* labels_host);
 
 /* Sec. 4.3: slices the monolithic cache along the head dimension into the Sink-Dummy buffer (one block per
  * head), the Global buffer and the Spatial buffer (full window each).  Needs labels and >= 1 cached block.
- * Allocates nothing (the buffers come from the arena reserved at create); frees the monolithic cache unless
- * keep_monolithic.  State becomes SPLIT. */
+ * Allocates nothing (the buffers come from the arena reserved at create); unless keep_monolithic, the monolithic
+ * cache is released in stream order after the gather (cudaFreeAsync: no host or device stall).  State becomes SPLIT. */
 int headcast_split_cache(headcast_ctx* ctx, void* stream);
 
 /* Sec. 4.4: head-specific attention of one block's queries, one launch for all pathways.  Sink heads read

@@ -15,6 +15,7 @@
 
 #include "attn_kernel.cuh"
 #include "copy_kernels.cuh"
+#include "move_kernels.cuh"
 #include "score_kernels.cuh"
 #include "tmap.h"
 
@@ -94,6 +95,17 @@ struct headcast_ctx {
   int32_t *sp_base = nullptr, *sp_nc = nullptr;
   CellGeom* cells_dev = nullptr;
   CUtensorMap maps[2 * N_MAP_PAIRS];  // host copies; every attention launch carries them as kernel parameters
+  // bulk tile movement (move_kernels.cuh): rectangles of the token grid per Spatial cell, their distinct box shapes,
+  // and the source tensor maps - of the monolithic cache (built at create) and of recently seen caller blocks
+  struct MoveShape { int cw, rows; };
+  struct MoveMaps { const void *k = nullptr, *v = nullptr; CUtensorMap rows[2], box[2][MOVE_MAX_SHAPES]; };
+  bool move_ok = false;     // false: the geometry does not fit the bulk path (very wide cells, too many cell shapes)
+  std::vector<MoveBox> move_boxes;
+  std::vector<MoveShape> move_shapes;
+  MoveBox* move_boxes_dev = nullptr;
+  MoveMaps move_mono;
+  MoveMaps move_recent[8];
+  int move_next = 0;
   int32_t* status_dev = nullptr;
 
   Schedule sched_dense, sched_hc, sched_cls, sched_proxy;
@@ -732,6 +744,115 @@ void fill_route(headcast_ctx* c, RouteParams& r) {
   }
 }
 
+// Source tensor maps of the bulk path for a [rows][H*d] tensor at k / v.
+bool build_move_maps(headcast_ctx* c, headcast_ctx::MoveMaps& m, const void* k, const void* v, uint64_t rows) {
+  const uint64_t row_elems = static_cast<uint64_t>(c->H) * c->D;
+  const uint32_t tile_rows = MOVE_STAGE_BYTES / (c->D * 2);
+  const void* base[2] = {k, v};
+  for (int kv = 0; kv < 2; ++kv) {
+    if (!make_tmap_bf16_rows(&m.rows[kv], base[kv], row_elems, rows, c->D, tile_rows)) return false;
+    for (size_t s = 0; s < c->move_shapes.size(); ++s)
+      if (!make_tmap_bf16_grid(&m.box[kv][s], base[kv], row_elems, rows, c->G_w, c->D, c->move_shapes[s].cw, c->move_shapes[s].rows))
+        return false;
+  }
+  m.k = k;
+  m.v = v;
+  return true;
+}
+
+// The same routing as route_block_kernel (RouteParams says which source block feeds which buffer), as bulk tile jobs.
+int launch_move(headcast_ctx* c, const RouteParams& r, int n_src, cudaStream_t st) {
+  static bool configured[64] = {};
+  int dev = 0;
+  HC_CUDA(c, cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64 || !configured[dev]) {
+    HC_CUDA(c, cudaFuncSetAttribute(move_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, MOVE_SMEM_BYTES));
+    if (dev >= 0 && dev < 64) configured[dev] = true;
+  }
+  MoveParams p;
+  std::memset(&p, 0, sizeof(p));
+  const headcast_ctx::MoveMaps* maps = nullptr;
+  if (r.src_stride != 0) {
+    maps = &c->move_mono;
+  } else {
+    for (auto& m : c->move_recent)
+      if (m.k == r.src_k && m.v == r.src_v && m.k) maps = &m;
+    if (!maps) {
+      headcast_ctx::MoveMaps& m = c->move_recent[c->move_next];
+      c->move_next = (c->move_next + 1) % 8;
+      m.k = m.v = nullptr;
+      if (!build_move_maps(c, m, r.src_k, r.src_v, c->L)) return fail(c, HC_ERR_CUDA, "cuTensorMapEncodeTiled failed for the block to append");
+      maps = &m;
+    }
+  }
+  std::memcpy(p.map_rows, maps->rows, sizeof(p.map_rows));
+  std::memcpy(p.map_box, maps->box, sizeof(p.map_box));
+  p.src_k = reinterpret_cast<const __nv_bfloat16*>(r.src_k);
+  p.src_v = reinterpret_cast<const __nv_bfloat16*>(r.src_v);
+  p.mono_k = reinterpret_cast<__nv_bfloat16*>(r.mono_k);
+  p.mono_v = reinterpret_cast<__nv_bfloat16*>(r.mono_v);
+  p.sd_k = reinterpret_cast<__nv_bfloat16*>(r.sd_k);
+  p.sd_v = reinterpret_cast<__nv_bfloat16*>(r.sd_v);
+  p.g_k = reinterpret_cast<__nv_bfloat16*>(r.g_k);
+  p.g_v = reinterpret_cast<__nv_bfloat16*>(r.g_v);
+  p.sp_k = reinterpret_cast<__nv_bfloat16*>(r.sp_k);
+  p.sp_v = reinterpret_cast<__nv_bfloat16*>(r.sp_v);
+  p.boxes = c->move_boxes_dev;
+  p.status = c->status_dev;
+  p.src_block_rows = r.src_stride ? c->L : 0;
+  p.n_boxes = static_cast<int32_t>(c->move_boxes.size());
+  p.L = c->L; p.H = c->H; p.D = c->D; p.F_b = c->F_b; p.G_h = c->G_h; p.G_w = c->G_w;
+  p.n_blocks = c->n_blk;
+  p.n_sink = r.n_sink;
+  p.sd_slots = r.sd_slots;
+  p.rows_per_tile = MOVE_STAGE_BYTES / (c->D * 2);
+  p.tiles_rm = (c->L + p.rows_per_tile - 1) / p.rows_per_tile;
+  p.copy_mono = r.copy_mono;
+  p.copy_window = r.copy_window;
+  const long long block_bytes = static_cast<long long>(c->L) * c->H * c->D * 2;
+  p.mono_chunks = r.copy_mono ? static_cast<int32_t>((block_bytes + MOVE_STAGE_BYTES - 1) / MOVE_STAGE_BYTES) : 0;
+  p.n_src = n_src;
+  for (int h = 0; h < c->H; ++h) {
+    p.cls[h] = r.cls[h];
+    p.idx[h] = r.idx[h];
+    if (r.cls[h] == CLS_SPATIAL && r.copy_window) p.sp[p.n_sp++] = static_cast<int8_t>(h);
+  }
+  for (int k = 0; k < 4; ++k)
+    for (int h = 0; h < c->H; ++h) {
+      const int cl = r.cls[h];
+      if ((cl == CLS_GLOBAL && r.copy_window) || (cl == CLS_SINK && (k == 0 || k == 2)) || (cl == CLS_DUMMY && (k == 1 || k == 2)))
+        p.rm[k][p.n_rm[k]++] = static_cast<int8_t>(h);
+    }
+  long long jobs = 0;
+  for (int i = 0; i < n_src; ++i) {
+    p.slots[i] = r.slots[i];
+    p.sd_slot_sink[i] = r.sd_slot_sink[i];
+    p.sd_slot_dummy[i] = r.sd_slot_dummy[i];
+    p.kind[i] = r.kind[i];
+    p.job_first[i] = static_cast<int32_t>(jobs);
+    jobs += 2ll * (static_cast<long long>(p.n_rm[p.kind[i]]) * p.tiles_rm + static_cast<long long>(p.n_sp) * p.F_b * p.n_boxes + p.mono_chunks);
+  }
+  p.job_first[n_src] = static_cast<int32_t>(jobs);
+  if (jobs == 0) return HC_OK;
+  if (jobs >= (1ll << 31)) return fail(c, HC_ERR_UNSUPPORTED, "too many tile jobs");
+  const int ctas = static_cast<int>(std::min<long long>(c->n_sm, (jobs + MOVE_ENGINES - 1) / MOVE_ENGINES));
+  cudaLaunchConfig_t lc;
+  std::memset(&lc, 0, sizeof(lc));
+  lc.gridDim = dim3(ctas);
+  lc.blockDim = dim3(MOVE_ENGINES * 32);
+  lc.dynamicSmemBytes = MOVE_SMEM_BYTES;
+  lc.stream = st;
+  cudaLaunchAttribute attr;
+  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;  // see the kernel: it waits for its predecessor itself
+  attr.val.programmaticStreamSerializationAllowed = 1;
+  lc.attrs = &attr;
+  lc.numAttrs = 1;
+  HC_CUDA(c, cudaLaunchKernelEx(&lc, move_kernel, p));
+  HC_CUDA(c, cudaGetLastError());
+  ++c->launches;
+  return HC_OK;
+}
+
 int launch_route(headcast_ctx* c, RouteParams& r, int n_src, cudaStream_t st) {
   // which heads each kind of source row feeds (see RouteParams::kind)
   for (int k = 0; k < 4; ++k) {
@@ -750,6 +871,7 @@ int launch_route(headcast_ctx* c, RouteParams& r, int n_src, cudaStream_t st) {
     max_kept = std::max<int>(max_kept, r.n_kept[r.kind[i]]);
   }
   if (max_kept == 0) return HC_OK;  // nothing to move (e.g. an append when every head is a Sink head)
+  if (c->move_ok) return launch_move(c, r, n_src, st);
   const int per_token = max_kept * r.chunks;  // <= 64 heads * 16 chunks = 1024
   const int tokens_per_iter = std::max(1, 256 / per_token);
   const int threads = tokens_per_iter * per_token;
@@ -837,6 +959,44 @@ static int init_host(headcast_ctx* c, const headcast_config* cfg, std::vector<in
         }
       tok_off += g.ch * g.cw;
     }
+  // bulk tile movement: every cell (or, for a cell larger than a stage, every band of its rows) is one rectangle of
+  // the token grid; rectangles of equal (width, rows) share a tensor map
+  const int stage_tokens = MOVE_STAGE_BYTES / (c->D * 2);
+  c->move_ok = true;
+  c->move_boxes.clear();
+  c->move_shapes.clear();
+  for (size_t ci = 0; ci < c->cells.size() && c->move_ok; ++ci) {
+    const CellGeom& g = c->cells[ci];
+    if (g.cw > stage_tokens || g.cw > 256) {
+      c->move_ok = false;
+      break;
+    }
+    const int rb = std::min(std::min(g.ch, 256), std::max(1, stage_tokens / g.cw));
+    int shape = -1;
+    for (size_t s = 0; s < c->move_shapes.size(); ++s)
+      if (c->move_shapes[s].cw == g.cw && c->move_shapes[s].rows == rb) shape = static_cast<int>(s);
+    if (shape < 0) {
+      if (c->move_shapes.size() == MOVE_MAX_SHAPES) {
+        c->move_ok = false;
+        break;
+      }
+      shape = static_cast<int>(c->move_shapes.size());
+      c->move_shapes.push_back({g.cw, rb});
+    }
+    for (int r0 = 0; r0 < g.ch; r0 += rb) {
+      MoveBox b;
+      b.y0 = g.y0 + r0;
+      b.x0 = g.x0;
+      b.cw = g.cw;
+      b.rows = std::min(rb, g.ch - r0);
+      b.shape = shape;
+      b.box_tokens = g.cw * rb;
+      b.cell_tok_off = c->cell_tok_off[ci];
+      b.nc = g.ch * g.cw;
+      b.first_tok = r0 * g.cw;
+      c->move_boxes.push_back(b);
+    }
+  }
   return HC_OK;
 }
 
@@ -885,14 +1045,17 @@ int headcast_create(const headcast_config* cfg, headcast_ctx** out) {
   const size_t mono_bytes = cache_elems(c, c->H) * sizeof(__nv_bfloat16);
   cudaError_t e = cudaSuccess;
   auto step = [&](cudaError_t r) { if (e == cudaSuccess) e = r; };
-  step(cudaMalloc(&c->mono_k, mono_bytes));
-  step(cudaMalloc(&c->mono_v, mono_bytes));
+  // the monolithic cache comes from the stream-ordered allocator, so that the split can release it in stream order
+  // (cudaFreeAsync) instead of stalling the host and the device in a cudaFree
+  step(cudaMallocAsync(reinterpret_cast<void**>(&c->mono_k), mono_bytes, nullptr));
+  step(cudaMallocAsync(reinterpret_cast<void**>(&c->mono_v), mono_bytes, nullptr));
   step(cudaMalloc(&c->arena_k, mono_bytes));
   step(cudaMalloc(&c->arena_v, mono_bytes));
   step(cudaMalloc(&c->sp_base, c->T_f * sizeof(int32_t)));
   step(cudaMalloc(&c->sp_nc, c->T_f * sizeof(int32_t)));
   step(cudaMalloc(&c->cells_dev, c->cells.size() * sizeof(CellGeom)));
   step(cudaMalloc(&c->status_dev, sizeof(int32_t)));
+  if (c->move_ok) step(cudaMalloc(&c->move_boxes_dev, std::max<size_t>(1, c->move_boxes.size()) * sizeof(MoveBox)));
   if (e == cudaSuccess) {
     step(cudaMemset(c->mono_k, 0, mono_bytes));
     step(cudaMemset(c->mono_v, 0, mono_bytes));
@@ -902,7 +1065,13 @@ int headcast_create(const headcast_config* cfg, headcast_ctx** out) {
     step(cudaMemcpy(c->sp_base, sp_base.data(), c->T_f * sizeof(int32_t), cudaMemcpyHostToDevice));
     step(cudaMemcpy(c->sp_nc, sp_nc.data(), c->T_f * sizeof(int32_t), cudaMemcpyHostToDevice));
     step(cudaMemcpy(c->cells_dev, c->cells.data(), c->cells.size() * sizeof(CellGeom), cudaMemcpyHostToDevice));
+    if (c->move_ok && !c->move_boxes.empty())
+      step(cudaMemcpy(c->move_boxes_dev, c->move_boxes.data(), c->move_boxes.size() * sizeof(MoveBox), cudaMemcpyHostToDevice));
   }
+  if (e == cudaSuccess && c->move_ok &&
+      !build_move_maps(c, c->move_mono, c->mono_k, c->mono_v, static_cast<uint64_t>(c->n_blk) * c->L))
+    c->move_ok = false;  // the per-thread copy kernel serves every geometry
+
   int rc = HC_OK;
   if (e != cudaSuccess) rc = (e == cudaErrorMemoryAllocation) ? HC_ERR_NOMEM : HC_ERR_CUDA;
   if (rc == HC_OK) rc = build_maps(c);
@@ -918,7 +1087,10 @@ int headcast_create(const headcast_config* cfg, headcast_ctx** out) {
 int headcast_destroy(headcast_ctx* c) {
   if (!c) return HC_OK;
   cudaDeviceSynchronize();
-  void* ptrs[] = {c->mono_k, c->mono_v, c->arena_k, c->arena_v, c->sp_base, c->sp_nc, c->cells_dev, c->status_dev};
+  if (c->mono_k) cudaFreeAsync(c->mono_k, nullptr);
+  if (c->mono_v) cudaFreeAsync(c->mono_v, nullptr);
+  cudaDeviceSynchronize();
+  void* ptrs[] = {c->arena_k, c->arena_v, c->sp_base, c->sp_nc, c->cells_dev, c->status_dev, c->move_boxes_dev};
   for (void* p : ptrs)
     if (p) cudaFree(p);
   if (c->ev_a) cudaEventDestroy(c->ev_a);
@@ -1224,10 +1396,9 @@ int headcast_split_cache(headcast_ctx* c, void* stream) {
     int rc = launch_route(c, r, static_cast<int>(c->slots.size()), st);
     if (rc != HC_OK) return rc;
   }
-  if (!c->cfg.keep_monolithic) {
-    HC_CUDA(c, cudaStreamSynchronize(st));
-    cudaFree(c->mono_k);
-    cudaFree(c->mono_v);
+  if (!c->cfg.keep_monolithic) {  // released in stream order, after the gather that reads it
+    HC_CUDA(c, cudaFreeAsync(c->mono_k, st));
+    HC_CUDA(c, cudaFreeAsync(c->mono_v, st));
     c->mono_k = c->mono_v = nullptr;
   }
   c->state = STATE_SPLIT;
