@@ -26,7 +26,7 @@ struct CellGeom {
   int32_t y0, x0, ch, cw;  // top-left grid position and extent of a deployed Spatial cell
 };
 
-enum : int32_t { OUT_BF16 = 0, OUT_PARTIAL = 1, OUT_F32_LSE = 2 };
+enum : int32_t { OUT_BF16 = 0, OUT_PARTIAL = 1 };
 
 struct WorkItem {
   int32_t head;           // original head index: addresses Q and the output
@@ -42,7 +42,7 @@ struct WorkItem {
   int32_t tile_begin;     // this item covers tiles [tile_begin, tile_end) of the segment-major enumeration
   int32_t tile_end;
   int32_t out_mode;       // OUT_*
-  int32_t out_slot;       // OUT_PARTIAL: partial slot; OUT_F32_LSE: pass index
+  int32_t out_slot;       // OUT_PARTIAL: partial slot
 };
 
 struct AttnParams {
@@ -54,8 +54,6 @@ struct AttnParams {
   float* part_o;           // [slot][256][d] unnormalised partial outputs
   float2* part_ml;         // [slot][256] (running max in the log2 domain, row sum)
   float* part_mid;         // [slot][256] Spatial proxy only: the part of the row sum that came from the middle blocks
-  float* f32_o;            // [pass][L][H][d] normalised fp32 outputs (classification)
-  float* f32_lse;          // [pass][L][H] natural-log LSE; Spatial proxy also writes [pass + 1] = middle-block LSE
   int32_t n_heads, tokens_per_frame, grid_w, block_tokens;
   float scale_log2e;       // softmax scale * log2(e)
   int32_t* status;
@@ -482,9 +480,7 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const __grid_cons
             dst[i] = o4;
           }
         } else {
-          float* base = (w.out_mode == OUT_PARTIAL)
-                            ? p.part_o + (static_cast<size_t>(w.out_slot) * 256 + t * 128 + r) * D + half * OC
-                            : p.f32_o + static_cast<size_t>(w.out_slot) * p.block_tokens * p.n_heads * D + row_elem;
+          float* base = p.part_o + (static_cast<size_t>(w.out_slot) * 256 + t * 128 + r) * D + half * OC;
           float4* dst = reinterpret_cast<float4*>(base + ch * 32);
 #pragma unroll
           for (int i = 0; i < 8; ++i)
@@ -492,17 +488,9 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const __grid_cons
                                  __uint_as_float(v[4 * i + 2]) * mult, __uint_as_float(v[4 * i + 3]) * mult);
         }
       }
-      if (row_valid && half == 0) {
-        if (w.out_mode == OUT_PARTIAL) {
-          p.part_ml[static_cast<size_t>(w.out_slot) * 256 + t * 128 + r] = make_float2(m_ref, l_sum);
-          if (PROXY) p.part_mid[static_cast<size_t>(w.out_slot) * 256 + t * 128 + r] = l_mid;
-        } else if (w.out_mode == OUT_F32_LSE) {
-          const float ln2 = 0.6931471805599453f;
-          const size_t lh = static_cast<size_t>(p.block_tokens) * p.n_heads;
-          const size_t idx = static_cast<size_t>(token) * p.n_heads + w.head;
-          p.f32_lse[w.out_slot * lh + idx] = (l_sum > 0.f) ? m_ref * ln2 + __logf(l_sum) : -INFINITY;
-          if (PROXY) p.f32_lse[(w.out_slot + 1) * lh + idx] = (l_mid > 0.f) ? m_ref * ln2 + __logf(l_mid) : -INFINITY;
-        }
+      if (row_valid && half == 0 && w.out_mode == OUT_PARTIAL) {
+        p.part_ml[static_cast<size_t>(w.out_slot) * 256 + t * 128 + r] = make_float2(m_ref, l_sum);
+        if (PROXY) p.part_mid[static_cast<size_t>(w.out_slot) * 256 + t * 128 + r] = l_mid;
       }
       if (p.trace && t == 0 && r == 0 && half == 0) p.trace[2 * it + 1] = global_timer_ns();
     }
@@ -559,118 +547,6 @@ combine_kernel(const CombineEntry* entries, const CellGeom* cells, const float* 
   o4.z = pack_bf16x2(acc[4] * inv, acc[5] * inv);
   o4.w = pack_bf16x2(acc[6] * inv, acc[7] * inv);
   *reinterpret_cast<uint4*>(out + (static_cast<size_t>(token) * n_heads + e.head) * D + c * 8) = o4;
-}
-
-// Classification: the reference attention (Eq. 2) and the Sink / Dummy proxies from ONE sweep over the keys.  The
-// sweep is cut into key ranges tagged first block / middle blocks / newest block, every range leaves an unnormalised
-// partial result, and this kernel merges them three ways per query row:
-//   all ranges -> reference output, pass 0;  first block only -> Sink proxy, pass 1;  newest block only -> Dummy
-//   proxy, pass 2;  each with its log-sum-exp (natural log).
-// parts[first_part .. first_part + n_parts) of a group list (partial slot, tag); a group is one 256-row query pair.
-struct ClsPart {
-  int32_t slot, tag;  // tag: 0 first block, 1 middle, 2 newest block
-};
-struct ClsGroup {
-  int32_t head, q_start, q_count[2], first_part, n_parts;
-};
-
-template <int D>
-__global__ void __launch_bounds__(COMBINE_ROWS * (D / 8))
-cls_combine_kernel(const ClsGroup* groups, const ClsPart* parts, const float* part_o, const float2* part_ml, float* f32_o,
-                   float* f32_lse, int n_heads, int block_tokens) {
-  constexpr int CHUNKS = D / 8;
-  constexpr int BLOCKS_PER_TILE = 128 / COMBINE_ROWS;
-  const ClsGroup g = groups[blockIdx.x / (2 * BLOCKS_PER_TILE)];
-  const int sub = (blockIdx.x / BLOCKS_PER_TILE) & 1;
-  const int r = (blockIdx.x % BLOCKS_PER_TILE) * COMBINE_ROWS + threadIdx.x / CHUNKS;
-  const int c = threadIdx.x % CHUNKS;
-  if (r >= g.q_count[sub]) return;
-  const ClsPart* pp = parts + g.first_part;
-  float m[3] = {-INFINITY, -INFINITY, -INFINITY};  // all, first, newest
-  for (int i = 0; i < g.n_parts; ++i) {
-    const float mi = part_ml[static_cast<size_t>(pp[i].slot) * 256 + sub * 128 + r].x;
-    m[0] = fmaxf(m[0], mi);
-    if (pp[i].tag == 0) m[1] = fmaxf(m[1], mi);
-    if (pp[i].tag == 2) m[2] = fmaxf(m[2], mi);
-  }
-  float acc[3][8], l[3] = {0.f, 0.f, 0.f};
-#pragma unroll
-  for (int k = 0; k < 3; ++k)
-#pragma unroll
-    for (int j = 0; j < 8; ++j) acc[k][j] = 0.f;
-  for (int i = 0; i < g.n_parts; ++i) {
-    const size_t row = static_cast<size_t>(pp[i].slot) * 256 + sub * 128 + r;
-    const float2 ml = part_ml[row];
-    if (ml.x == -INFINITY) continue;
-    const float4* src = reinterpret_cast<const float4*>(part_o + row * D + c * 8);
-    const float4 a = src[0], b = src[1];
-    const float v[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
-#pragma unroll
-    for (int k = 0; k < 3; ++k) {
-      const bool in_set = (k == 0) || (k == 1 && pp[i].tag == 0) || (k == 2 && pp[i].tag == 2);
-      if (!in_set) continue;
-      const float wgt = ex2_approx(ml.x - m[k]);
-      l[k] += wgt * ml.y;
-#pragma unroll
-      for (int j = 0; j < 8; ++j) acc[k][j] += wgt * v[j];
-    }
-  }
-  const int token = g.q_start + sub * 128 + r;
-  const size_t lh = static_cast<size_t>(block_tokens) * n_heads;
-  const size_t idx = static_cast<size_t>(token) * n_heads + g.head;
-  const float ln2 = 0.6931471805599453f;
-#pragma unroll
-  for (int k = 0; k < 3; ++k) {
-    const float inv = l[k] > 0.f ? 1.f / l[k] : 0.f;
-    float4* dst = reinterpret_cast<float4*>(f32_o + (k * lh + idx) * D + c * 8);
-    dst[0] = make_float4(acc[k][0] * inv, acc[k][1] * inv, acc[k][2] * inv, acc[k][3] * inv);
-    dst[1] = make_float4(acc[k][4] * inv, acc[k][5] * inv, acc[k][6] * inv, acc[k][7] * inv);
-    if (c == 0) f32_lse[k * lh + idx] = (l[k] > 0.f) ? m[k] * ln2 + __logf(l[k]) : -INFINITY;
-  }
-}
-
-// Classification, Spatial proxy: the band of one query pair may be cut into pieces along its key range like any other
-// item; this merges the pieces into the proxy output (pass `pass`), its log-sum-exp (plane `pass`) and the
-// log-sum-exp of the middle blocks' share (plane `pass` + 1).
-template <int D>
-__global__ void __launch_bounds__(COMBINE_ROWS * (D / 8))
-proxy_combine_kernel(const ClsGroup* groups, const ClsPart* parts, const float* part_o, const float2* part_ml,
-                     const float* part_mid, float* f32_o, float* f32_lse, int n_heads, int block_tokens, int pass) {
-  constexpr int CHUNKS = D / 8;
-  constexpr int BLOCKS_PER_TILE = 128 / COMBINE_ROWS;
-  const ClsGroup g = groups[blockIdx.x / (2 * BLOCKS_PER_TILE)];
-  const int sub = (blockIdx.x / BLOCKS_PER_TILE) & 1;
-  const int r = (blockIdx.x % BLOCKS_PER_TILE) * COMBINE_ROWS + threadIdx.x / CHUNKS;
-  const int c = threadIdx.x % CHUNKS;
-  if (r >= g.q_count[sub] || g.n_parts == 0) return;  // a band left whole has written its output itself
-  const ClsPart* pp = parts + g.first_part;
-  float m = -INFINITY;
-  for (int i = 0; i < g.n_parts; ++i) m = fmaxf(m, part_ml[static_cast<size_t>(pp[i].slot) * 256 + sub * 128 + r].x);
-  float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0}, l = 0.f, l_mid = 0.f;
-  for (int i = 0; i < g.n_parts; ++i) {
-    const size_t row = static_cast<size_t>(pp[i].slot) * 256 + sub * 128 + r;
-    const float2 ml = part_ml[row];
-    if (ml.x == -INFINITY) continue;
-    const float wgt = ex2_approx(ml.x - m);
-    l += wgt * ml.y;
-    l_mid += wgt * part_mid[row];
-    const float4* src = reinterpret_cast<const float4*>(part_o + row * D + c * 8);
-    const float4 a = src[0], b = src[1];
-    acc[0] += wgt * a.x; acc[1] += wgt * a.y; acc[2] += wgt * a.z; acc[3] += wgt * a.w;
-    acc[4] += wgt * b.x; acc[5] += wgt * b.y; acc[6] += wgt * b.z; acc[7] += wgt * b.w;
-  }
-  const int token = g.q_start + sub * 128 + r;
-  const size_t lh = static_cast<size_t>(block_tokens) * n_heads;
-  const size_t idx = static_cast<size_t>(token) * n_heads + g.head;
-  const float ln2 = 0.6931471805599453f;
-  const float inv = l > 0.f ? 1.f / l : 0.f;
-  float4* dst = reinterpret_cast<float4*>(f32_o + (pass * lh + idx) * D + c * 8);
-  dst[0] = make_float4(acc[0] * inv, acc[1] * inv, acc[2] * inv, acc[3] * inv);
-  dst[1] = make_float4(acc[4] * inv, acc[5] * inv, acc[6] * inv, acc[7] * inv);
-  if (c == 0) {
-    f32_lse[pass * lh + idx] = (l > 0.f) ? m * ln2 + __logf(l) : -INFINITY;
-    f32_lse[(pass + 1) * lh + idx] = (l_mid > 0.f) ? m * ln2 + __logf(l_mid) : -INFINITY;
-  }
 }
 
 }  // namespace hc

@@ -213,7 +213,6 @@ struct Proto {  // one (head, query-tile pair, key range) before it is cut into 
   int n_tiles;
   int cls_group = -1;  // classification: every piece writes a partial result that belongs to this group ...
   int cls_tag = 0;     // ... with this tag (0 first block, 1 middle blocks, 2 newest block)
-  bool whole_is_final = false;  // ... unless the item stays in one piece, which then writes its own output mode
 };
 
 // Query-tile pairs of rows [q_lo, q_hi) (q_lo a multiple of 256; by default all rows) of one head and key range.
@@ -331,13 +330,13 @@ void finalize_schedule(headcast_ctx* c, Schedule& s, std::vector<Proto>& protos,
           w.tile_begin = begin;
           w.tile_end = begin + take;
           parts.push_back(std::make_pair(cta, w));
-          const bool cut = (take < left) || begin > 0 || (p.cls_group >= 0 && !p.whole_is_final);
+          const bool cut = (take < left) || begin > 0 || (p.cls_group >= 0);
           const double cost = per_tile * take + overhead + (cut ? PARTIAL_EXTRA : 0.0);
           room -= cost;
           if (cta == n_cta - 1) last_load += cost;
           begin += take;
         }
-        if (p.cls_group >= 0 && !(p.whole_is_final && parts.size() == 1)) {
+        if (p.cls_group >= 0) {
           for (auto& pr : parts) {
             pr.second.out_mode = OUT_PARTIAL;
             pr.second.out_slot = s.n_slots++;
@@ -635,8 +634,6 @@ int run_schedule(headcast_ctx* c, Schedule& s, const void* q, void* out, bool pr
   p.part_o = c->part_o.ptr;
   p.part_ml = c->part_ml.ptr;
   p.part_mid = c->part_mid.ptr;
-  p.f32_o = c->cls_o.ptr;
-  p.f32_lse = c->cls_lse.ptr;
   p.n_heads = c->H;
   p.tokens_per_frame = c->T_f;
   p.grid_w = c->G_w;
@@ -665,26 +662,25 @@ int run_schedule(headcast_ctx* c, Schedule& s, const void* q, void* out, bool pr
   else
     rc = proxy ? launch_attn_t<64, true>(c, p, st) : launch_attn_t<64, false>(c, p, st);
   if (rc != HC_OK) return rc;
-  if (!s.cls_groups.empty() && proxy) {
+  if (!s.cls_groups.empty()) {
+    // classification: merge the pieces of every query pair and score its rows (score_kernels.cuh)
     const unsigned blocks = static_cast<unsigned>(s.cls_groups.size()) * 2 * (128 / COMBINE_ROWS);
-    if (c->D == 128)
-      proxy_combine_kernel<128><<<blocks, COMBINE_ROWS * 16, 0, st>>>(s.cls_groups_dev.ptr, s.cls_parts_dev.ptr, c->part_o.ptr,
-                                                                      c->part_ml.ptr, c->part_mid.ptr, c->cls_o.ptr,
-                                                                      c->cls_lse.ptr, c->H, c->L, 3);
-    else
-      proxy_combine_kernel<64><<<blocks, COMBINE_ROWS * 8, 0, st>>>(s.cls_groups_dev.ptr, s.cls_parts_dev.ptr, c->part_o.ptr,
-                                                                    c->part_ml.ptr, c->part_mid.ptr, c->cls_o.ptr,
-                                                                    c->cls_lse.ptr, c->H, c->L, 3);
-    HC_CUDA(c, cudaGetLastError());
-    ++c->launches;
-  } else if (!s.cls_groups.empty()) {
-    const unsigned blocks = static_cast<unsigned>(s.cls_groups.size()) * 2 * (128 / COMBINE_ROWS);
-    if (c->D == 128)
-      cls_combine_kernel<128><<<blocks, COMBINE_ROWS * 16, 0, st>>>(s.cls_groups_dev.ptr, s.cls_parts_dev.ptr, c->part_o.ptr,
-                                                                    c->part_ml.ptr, c->cls_o.ptr, c->cls_lse.ptr, c->H, c->L);
-    else
-      cls_combine_kernel<64><<<blocks, COMBINE_ROWS * 8, 0, st>>>(s.cls_groups_dev.ptr, s.cls_parts_dev.ptr, c->part_o.ptr,
-                                                                  c->part_ml.ptr, c->cls_o.ptr, c->cls_lse.ptr, c->H, c->L);
+    const unsigned threads = COMBINE_ROWS * (c->D / 8);
+    if (proxy) {
+      if (c->D == 128)
+        proxy_combine_kernel<128><<<blocks, threads, 0, st>>>(s.cls_groups_dev.ptr, s.cls_parts_dev.ptr, c->part_o.ptr, c->part_ml.ptr,
+                                                              c->part_mid.ptr, c->cls_o.ptr, c->cls_lse.ptr, c->cls_tok.ptr, c->H, c->L);
+      else
+        proxy_combine_kernel<64><<<blocks, threads, 0, st>>>(s.cls_groups_dev.ptr, s.cls_parts_dev.ptr, c->part_o.ptr, c->part_ml.ptr,
+                                                             c->part_mid.ptr, c->cls_o.ptr, c->cls_lse.ptr, c->cls_tok.ptr, c->H, c->L);
+    } else {
+      if (c->D == 128)
+        cls_combine_kernel<128><<<blocks, threads, 0, st>>>(s.cls_groups_dev.ptr, s.cls_parts_dev.ptr, c->part_o.ptr, c->part_ml.ptr,
+                                                            c->cls_o.ptr, c->cls_lse.ptr, c->cls_tok.ptr, c->H, c->L);
+      else
+        cls_combine_kernel<64><<<blocks, threads, 0, st>>>(s.cls_groups_dev.ptr, s.cls_parts_dev.ptr, c->part_o.ptr, c->part_ml.ptr,
+                                                           c->cls_o.ptr, c->cls_lse.ptr, c->cls_tok.ptr, c->H, c->L);
+    }
     HC_CUDA(c, cudaGetLastError());
     ++c->launches;
   }
@@ -1211,8 +1207,8 @@ int headcast_classify(headcast_ctx* c, const void* q, int32_t* labels_host, floa
   if (n_filled(c) < 2) return fail(c, HC_ERR_STATE, "classification needs at least two cached blocks");
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const size_t rows = static_cast<size_t>(c->L) * c->H;
-  HC_CUDA(c, c->cls_o.reserve(4 * rows * c->D));
-  HC_CUDA(c, c->cls_lse.reserve(5 * rows));
+  HC_CUDA(c, c->cls_o.reserve(rows * c->D));  // the reference output (fp32); the proxy outputs never leave registers
+  HC_CUDA(c, c->cls_lse.reserve(rows));
   HC_CUDA(c, c->cls_tok.reserve(TOK_N * rows));
   HC_CUDA(c, c->cls_scores.reserve(static_cast<size_t>(c->H) * HC_N_SCORES));
   HC_CUDA(c, c->cls_labels.reserve(c->H));
@@ -1281,8 +1277,6 @@ int headcast_classify(headcast_ctx* c, const void* q, int32_t* labels_host, floa
         }
         WorkItem w = range_item(h, MAP_MONO, h * c->D, a, b - a);
         w.seg_stride = c->T_f;
-        w.out_mode = OUT_F32_LSE;
-        w.out_slot = 3;
         Proto p;
         p.w = w;
         p.w.q_start[0] = q0;
@@ -1292,7 +1286,7 @@ int headcast_classify(headcast_ctx* c, const void* q, int32_t* labels_host, floa
         p.n_tiles = w.tiles_per_seg * n_filled(c) * c->F_b;
         p.w.tile_begin = 0;
         p.w.tile_end = p.n_tiles;
-        // a band cut into pieces writes partial results, which proxy_combine_kernel merges
+        // whole or cut into pieces, a band leaves partial results that proxy_combine_kernel merges and scores
         ClsGroup g;
         g.head = h;
         g.q_start = q0;
@@ -1302,7 +1296,6 @@ int headcast_classify(headcast_ctx* c, const void* q, int32_t* labels_host, floa
         g.n_parts = 0;
         p.cls_group = static_cast<int>(c->sched_proxy.cls_groups.size());
         p.cls_tag = 0;
-        p.whole_is_final = true;
         c->sched_proxy.cls_groups.push_back(g);
         protos.push_back(p);
       }
@@ -1312,14 +1305,6 @@ int headcast_classify(headcast_ctx* c, const void* q, int32_t* labels_host, floa
   rc = run_schedule(c, c->sched_proxy, q, nullptr, true, st);
   if (rc != HC_OK) return rc;
   {
-    const long long warps = static_cast<long long>(rows);
-    const unsigned blocks = static_cast<unsigned>((warps * 32 + 255) / 256);
-    if (c->D == 128)
-      token_scores_kernel<128><<<blocks, 256, 0, st>>>(c->cls_o.ptr, c->cls_lse.ptr, c->cls_tok.ptr, c->L, c->H);
-    else
-      token_scores_kernel<64><<<blocks, 256, 0, st>>>(c->cls_o.ptr, c->cls_lse.ptr, c->cls_tok.ptr, c->L, c->H);
-    HC_CUDA(c, cudaGetLastError());
-    ++c->launches;
     DecideParams d;
     d.tok = c->cls_tok.ptr;
     d.scores = c->cls_scores.ptr;
@@ -1337,7 +1322,7 @@ int headcast_classify(headcast_ctx* c, const void* q, int32_t* labels_host, floa
     d.gamma = c->cfg.gamma;
     d.rule = c->cfg.rule;
     d.mass_tau = c->cfg.mass_tau;
-    head_decide_kernel<<<c->H, 512, 0, st>>>(d);
+    head_decide_kernel<<<c->H, 1024, 0, st>>>(d);
     HC_CUDA(c, cudaGetLastError());
     ++c->launches;
   }
