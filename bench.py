@@ -612,7 +612,7 @@ def measure_workload(w, args, torch, HeadCast, peaks, dist, local, e2e_leg: bool
 
     # ---- sustained leg: the same steps for >= 2 s of GPU time, so that the clock sampler sees the clocks the kernel
     # settles at under the power cap; the figure that compares workloads run at different clocks is FLOP per SM clock
-    n_sus = int(min(20000, max(args.steps, 2000.0 / max(res["ms_per_step"], 1e-3))))
+    n_sus = 4 if args.no_sustained else int(min(20000, max(args.steps, 2000.0 / max(res["ms_per_step"], 1e-3))))
     sus_kernel = []
     with ClockSampler(local) as sus_clocks:
         for i in range(n_sus):
@@ -778,6 +778,7 @@ def main():
                          "a short run for profiler captures of the copy kernel")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-phases", action="store_true")
+    ap.add_argument("--no-sustained", action="store_true", help="skip the >= 2 s sustained leg (short runs for profiler captures)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     if args.workload == "rollout":

@@ -211,6 +211,10 @@ int build_maps(headcast_ctx* c) {
 struct Proto {  // one (head, query-tile pair, key range) before it is cut into parts
   WorkItem w;
   int n_tiles;
+  int tile_off = 0;  // first tile of this proto inside the key sweep (key chunks of a long stream; else 0)
+  int group = -1;    // pieces with the same group id are partial results of one query-tile pair (assigned in finalize_schedule)
+  int phase = -1;    // phase this proto is placed in (-1: the last line)
+  bool always_partial = false;  // one of several key chunks of its pair: never a final result on its own
   int cls_group = -1;  // classification: every piece writes a partial result that belongs to this group ...
   int cls_tag = 0;     // ... with this tag (0 first block, 1 middle blocks, 2 newest block)
 };
@@ -306,7 +310,6 @@ void finalize_schedule(headcast_ctx* c, Schedule& s, std::vector<Proto>& protos,
       };
       for (size_t pi = first_proto; pi < last_proto; ++pi) {
         const Proto& p = protos[pi];
-        const int n_q = p.w.q_count[1] > 0 ? 2 : 1;
         const double per_tile = tile_cost(p.w), overhead = item_overhead(p.w);
         std::vector<std::pair<int, WorkItem>> parts;  // (cta, piece)
         int begin = 0;
@@ -327,10 +330,10 @@ void finalize_schedule(headcast_ctx* c, Schedule& s, std::vector<Proto>& protos,
                // tiles, or a share smaller than one piece): it takes the rest whole
           }
           WorkItem w = p.w;
-          w.tile_begin = begin;
-          w.tile_end = begin + take;
+          w.tile_begin = p.tile_off + begin;
+          w.tile_end = p.tile_off + begin + take;
           parts.push_back(std::make_pair(cta, w));
-          const bool cut = (take < left) || begin > 0 || (p.cls_group >= 0);
+          const bool cut = (take < left) || begin > 0 || (p.cls_group >= 0) || p.always_partial;
           const double cost = per_tile * take + overhead + (cut ? PARTIAL_EXTRA : 0.0);
           room -= cost;
           if (cta == n_cta - 1) last_load += cost;
@@ -345,27 +348,13 @@ void finalize_schedule(headcast_ctx* c, Schedule& s, std::vector<Proto>& protos,
           }
           continue;
         }
-        if (parts.size() == 1) {
-          bins[parts[0].first].push_back(parts[0].second);
-          continue;
-        }
-        const int first_slot = s.n_slots;
+        // pieces of ordinary items: whether a piece is a final or a partial result, and its slot, is settled once every
+        // phase is placed (the pieces of one query-tile pair may come from several key chunks); until then out_slot
+        // carries the pair's group id
         for (auto& pr : parts) {
           pr.second.out_mode = OUT_PARTIAL;
-          pr.second.out_slot = s.n_slots++;
+          pr.second.out_slot = p.group;
           bins[pr.first].push_back(pr.second);
-        }
-        for (int t = 0; t < n_q; ++t) {
-          CombineEntry e;
-          e.head = p.w.head;
-          e.cell = p.w.cell;
-          e.q_start = p.w.q_start[t];
-          e.q_count = p.w.q_count[t];
-          e.first_slot = first_slot;
-          e.n_parts = static_cast<int32_t>(parts.size());
-          e.sub = t;
-          e.pad = 0;
-          s.combine.push_back(e);
         }
       }
       return last_load;
@@ -425,18 +414,28 @@ void finalize_schedule(headcast_ctx* c, Schedule& s, std::vector<Proto>& protos,
     // Everything else (short streams, Spatial cells) follows in one last line.  Measured: 9-13 % off the 720P and
     // 1080P attention and dense sweeps, 6 % off the 480P dense sweep; at 480P the three Global heads (50 MB) are
     // left in one line, where phases only add partial results to merge.
+    // A stream too long for that on its own (1080P: 88 MB of K/V per Global head) is ALSO cut along its keys into
+    // chunks of at most HC_CHUNK_BYTES, every chunk a phase of its own: all CTAs sweep the same ~30 MB of keys at the
+    // same time, each query-tile pair leaves one partial result per chunk, and combine_kernel merges them.  Without the
+    // chunks the CTAs sit at 148 different places of the sweep, the whole stream is the working set, and 8.4x the
+    // algorithmic bytes came from DRAM at 1080P (ncu: 6.97 GB per launch).
     {
-      constexpr long long HC_PHASE_BYTES = 60ll << 20;
-      struct Stream { int map, head, phase; double cost; long long bytes; };
+      constexpr long long HC_PHASE_BYTES = 60ll << 20, HC_CHUNK_BYTES = 30ll << 20;
+      for (size_t pi = 0; pi < protos.size(); ++pi)
+        if (protos[pi].group < 0) protos[pi].group = static_cast<int>(pi);
+      struct Stream { int map, head, phase, n_chunks; double cost; long long bytes; };
       std::vector<Stream> streams;
       double all_cost = 0.0;
+      auto stream_of = [&](const Proto& p) {
+        return std::find_if(streams.begin(), streams.end(), [&](const Stream& st) { return st.map == p.w.kv_map && st.head == p.w.head; });
+      };
       for (const Proto& p : protos) {
         all_cost += item_cost(p.w);
         if (p.w.cell >= 0) continue;
-        auto it = std::find_if(streams.begin(), streams.end(), [&](const Stream& st) { return st.map == p.w.kv_map && st.head == p.w.head; });
+        auto it = stream_of(p);
         if (it == streams.end()) {
           const long long segs = (p.n_tiles + p.w.tiles_per_seg - 1) / p.w.tiles_per_seg;
-          streams.push_back({p.w.kv_map, p.w.head, -1, 0.0, segs * p.w.seg_len * c->D * 4ll});
+          streams.push_back({p.w.kv_map, p.w.head, -1, 1, 0.0, segs * p.w.seg_len * c->D * 4ll});
           it = streams.end() - 1;
         }
         it->cost += item_cost(p.w);
@@ -449,6 +448,17 @@ void finalize_schedule(headcast_ctx* c, Schedule& s, std::vector<Proto>& protos,
       for (Stream& st : streams) {
         if (st.cost < 20.0 * n_cta) continue;
         long_bytes += st.bytes;
+        // key chunks only for plain row ranges (one segment) that are not part of a classification sweep
+        const int chunks = static_cast<int>((st.bytes + HC_CHUNK_BYTES - 1) / HC_CHUNK_BYTES);
+        if (st.bytes > HC_PHASE_BYTES && s.cls_groups.empty() && st.cost / chunks >= 60.0 * n_cta) {
+          st.n_chunks = chunks;
+          st.phase = static_cast<int>(phase_bytes.size());
+          for (int k = 0; k < chunks; ++k) {
+            phase_bytes.push_back(HC_PHASE_BYTES);  // closed to other streams
+            phase_cost.push_back(st.cost / chunks);
+          }
+          continue;
+        }
         size_t ph = 0;
         while (ph < phase_bytes.size() && phase_bytes[ph] + st.bytes > HC_PHASE_BYTES) ++ph;
         if (ph == phase_bytes.size()) {
@@ -461,14 +471,38 @@ void finalize_schedule(headcast_ctx* c, Schedule& s, std::vector<Proto>& protos,
       }
       size_t done = 0;
       if (long_bytes > (64ll << 20) && all_cost >= 120.0 * n_cta) {  // below that the streams share L2 anyway (480P: 50 MB)
+        // every proto learns its phase; protos of a chunked stream are replaced by one proto per key chunk
+        std::vector<Proto> expanded;
+        expanded.reserve(protos.size());
+        for (const Proto& p : protos) {
+          auto it = (p.w.cell >= 0) ? streams.end() : stream_of(p);
+          if (it == streams.end() || it->phase < 0) {
+            expanded.push_back(p);
+            continue;
+          }
+          if (it->n_chunks == 1 || p.w.seg_stride != 0 || p.n_tiles < 2 * it->n_chunks * MIN_PART_TILES) {
+            Proto q = p;
+            q.phase = it->phase;
+            expanded.push_back(q);
+            continue;
+          }
+          for (int k = 0; k < it->n_chunks; ++k) {
+            Proto q = p;
+            const int lo = static_cast<int>(static_cast<long long>(p.n_tiles) * k / it->n_chunks);
+            const int hi = static_cast<int>(static_cast<long long>(p.n_tiles) * (k + 1) / it->n_chunks);
+            q.tile_off = p.tile_off + lo;
+            q.n_tiles = hi - lo;
+            q.w.tile_begin = q.tile_off;
+            q.w.tile_end = q.tile_off + q.n_tiles;
+            q.phase = it->phase + k;
+            q.always_partial = true;
+            expanded.push_back(q);
+          }
+        }
+        protos.swap(expanded);
         for (size_t ph = 0; ph < phase_cost.size(); ++ph) {
           if (phase_cost[ph] < 60.0 * n_cta) continue;
-          auto in_phase = [&](const Proto& p) {
-            if (p.w.cell >= 0) return false;
-            for (const Stream& st : streams)
-              if (st.map == p.w.kv_map && st.head == p.w.head) return st.phase == static_cast<int>(ph);
-            return false;
-          };
+          auto in_phase = [&](const Proto& p) { return p.phase == static_cast<int>(ph); };
           auto mid = std::stable_partition(protos.begin() + done, protos.end(), in_phase);
           const size_t next = static_cast<size_t>(mid - protos.begin());
           if (next > done) place(done, next);
@@ -476,6 +510,45 @@ void finalize_schedule(headcast_ctx* c, Schedule& s, std::vector<Proto>& protos,
         }
       }
       if (done < protos.size() || protos.empty()) place(done, protos.size());
+    }
+    // ordinary items: the pieces of one query-tile pair (same group id, parked in out_slot) become a final result if
+    // there is only one, else partial results in consecutive slots, in key order, plus one merge entry per query tile
+    if (s.cls_groups.empty()) {
+      struct Piece { int bin, pos, tile_begin; };
+      std::vector<std::vector<Piece>> by_group;
+      for (int b = 0; b < n_cta; ++b)
+        for (size_t i = 0; i < bins[b].size(); ++i) {
+          const WorkItem& w = bins[b][i];
+          if (static_cast<size_t>(w.out_slot) >= by_group.size()) by_group.resize(w.out_slot + 1);
+          by_group[w.out_slot].push_back({b, static_cast<int>(i), w.tile_begin});
+        }
+      s.combine.clear();
+      s.n_slots = 0;
+      for (auto& pieces : by_group) {
+        if (pieces.empty()) continue;
+        if (pieces.size() == 1) {
+          WorkItem& w = bins[pieces[0].bin][pieces[0].pos];
+          w.out_mode = OUT_BF16;
+          w.out_slot = 0;
+          continue;
+        }
+        std::sort(pieces.begin(), pieces.end(), [](const Piece& a, const Piece& b) { return a.tile_begin < b.tile_begin; });
+        const int first_slot = s.n_slots;
+        for (const Piece& pc : pieces) bins[pc.bin][pc.pos].out_slot = s.n_slots++;
+        const WorkItem& w0 = bins[pieces[0].bin][pieces[0].pos];
+        for (int t = 0; t < (w0.q_count[1] > 0 ? 2 : 1); ++t) {
+          CombineEntry e;
+          e.head = w0.head;
+          e.cell = w0.cell;
+          e.q_start = w0.q_start[t];
+          e.q_count = w0.q_count[t];
+          e.first_slot = first_slot;
+          e.n_parts = static_cast<int32_t>(pieces.size());
+          e.sub = t;
+          e.pad = 0;
+          s.combine.push_back(e);
+        }
+      }
     }
     // classification: the pieces of every group, in group order
     std::stable_sort(cls_raw.begin(), cls_raw.end(), [](const RawPart& a, const RawPart& b) { return a.group < b.group; });

@@ -113,6 +113,32 @@ def test_paper_workloads_are_covered_and_balanced(res):
         assert per_cta.max() <= 1.06 * per_cta.mean(), (res, dense, per_cta.max() / per_cta.mean())
 
 
+def test_long_key_streams_are_swept_chunk_by_chunk_by_all_ctas():
+    """1080P: one Global head's K/V (88 MB) does not fit L2 next to everything else, so its sweep is cut into key
+    chunks of at most 30 MB and every CTA works through the chunks in the same order: what the CTAs read at the same
+    time stays a fraction of L2."""
+    w = synth.wan("1080p")
+    items, first = binding.plan_schedule(config_of(w), list(w.labels), w.n_blocks, 148)
+    tile_bytes = 128 * w.head_dim * 2 * 2  # one key tile of K and V
+    for h in [i for i, lab in enumerate(w.labels) if lab == orc.GLOBAL]:
+        mine = items[:, F["head"]] == h
+        total_tiles = int(items[mine][0][F["tiles_per_seg"]])
+        n_chunks = -(-total_tiles * tile_bytes // (30 << 20))
+        assert n_chunks == 3
+        bounds = [total_tiles * k // n_chunks for k in range(n_chunks + 1)]
+        chunk_of = lambda it: next(k for k in range(n_chunks) if bounds[k] <= it[F["tile_begin"]] < bounds[k + 1])
+        busy = 0
+        for b in range(148):
+            seq = [chunk_of(it) for it in items[first[b]:first[b + 1]] if it[F["head"]] == h]
+            for it in items[first[b]:first[b + 1]]:
+                if it[F["head"]] == h:  # no piece straddles a chunk boundary
+                    k = chunk_of(it)
+                    assert bounds[k] <= it[F["tile_begin"]] < it[F["tile_end"]] <= bounds[k + 1]
+            assert seq == sorted(seq)
+            busy += len(set(seq)) == n_chunks
+        assert busy >= 140  # (nearly) every CTA takes part in every chunk
+
+
 def test_growth_phase_and_odd_cta_counts():
     w = synth.small()
     for n_filled in (1, 2, 4):
