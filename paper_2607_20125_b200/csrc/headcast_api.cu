@@ -420,7 +420,13 @@ void finalize_schedule(headcast_ctx* c, Schedule& s, std::vector<Proto>& protos,
     // chunks the CTAs sit at 148 different places of the sweep, the whole stream is the working set, and 8.4x the
     // algorithmic bytes came from DRAM at 1080P (ncu: 6.97 GB per launch).
     {
-      constexpr long long HC_PHASE_BYTES = 60ll << 20, HC_CHUNK_BYTES = 30ll << 20;
+#ifndef HC_PHASE_MB
+#define HC_PHASE_MB 60
+#endif
+#ifndef HC_CHUNK_MB
+#define HC_CHUNK_MB 30
+#endif
+      constexpr long long HC_PHASE_BYTES = static_cast<long long>(HC_PHASE_MB) << 20, HC_CHUNK_BYTES = static_cast<long long>(HC_CHUNK_MB) << 20;
       for (size_t pi = 0; pi < protos.size(); ++pi)
         if (protos[pi].group < 0) protos[pi].group = static_cast<int>(pi);
       struct Stream { int map, head, phase, n_chunks; double cost; long long bytes; };
