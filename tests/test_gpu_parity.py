@@ -131,6 +131,33 @@ def test_archetype_groups_may_be_empty(labels):
     run_pipeline(w, fill=3, extra=1, labels=labels)
 
 
+@pytest.mark.parametrize("d,cell_h,cell_w", [(128, 13, 11), (64, 13, 22), (128, 2, 3)])
+def test_copy_path_geometries_bands_of_large_cells_and_many_small_cells(d, cell_h, cell_w):
+    # the bulk copy kernel moves a Spatial cell as one box of the token grid - or, for a cell with more tokens than a
+    # 32 KB stage holds, in bands of its rows (13 x 11 tokens at d = 128: bands of 11 + 2 rows; 13 x 22 at d = 64: 11 + 2);
+    # 2 x 3 cells give 42 small boxes per frame.  Split during growth, appends through two rolls, refresh of the newest
+    # block, Sink / Dummy heads in both modes: exported caches bit-exact every time, attention against the oracle.
+    for sd_mode in (0, 1):
+        w = synth.small(head_dim=d, cell_h=cell_h, cell_w=cell_w)
+        p = Pair(w, keep_monolithic=(sd_mode == 0), sd_mode=sd_mode)
+        p.append(2)
+        p.check_cache()
+        p.hc.set_labels(w.labels)
+        p.hc.split_cache()
+        p.cache.split(w.labels)
+        p.check_cache()
+        for i in range(4):
+            p.append()
+            p.check_cache()
+            if i == 1:
+                p.overwrite_last(i)
+                p.check_cache()
+        p.check_attention(dense=False)
+        if sd_mode == 0:
+            p.check_attention(dense=True)
+        p.hc.destroy()
+
+
 def test_explicit_cell_edges_one_row_cells():
     w = synth.small(n_blocks=3)
     rows_e = [0, 1, 2, 7, 13]
