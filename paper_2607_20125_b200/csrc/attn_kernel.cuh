@@ -320,15 +320,25 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const __grid_cons
         token = w.q_start[t] + r;
         if (w.cell >= 0) token = cell_query_token(p.cells[w.cell], token, p.tokens_per_frame, p.grid_w);
       }
-      // ---- stage this thread's half of its query row into shared memory (swizzled); invalid rows are zero
+      // ---- stage this warp's 32 query rows (its half of the columns) into shared memory (swizzled); invalid rows are
+      // zero.  The lanes share the rows: CH consecutive lanes fetch the CH 16-byte chunks of one row, so a load
+      // instruction touches 32 / CH rows (4 lines of 128 bytes at d = 128) instead of 32 - with one row per lane the
+      // 16 warps needed 4096 line visits per item and the load/store unit, not the latency, set the time (2.5 us).
       {
-        const uint4* src = reinterpret_cast<const uint4*>(p.q + (static_cast<size_t>(token) * p.n_heads + w.head) * D);
+        constexpr int CH = D / 16;  // 16-byte chunks of a half row
+        uint4 v[CH];
 #pragma unroll
-        for (int cc = 0; cc < D / 16; ++cc) {
-          const int c = half * (D / 16) + cc;
-          uint4 v = make_uint4(0, 0, 0, 0);
-          if (row_valid) v = __ldg(src + c);
-          *reinterpret_cast<uint4*>(sq + (c / 8) * SM::BLOCK_BYTES + sw128_offset(r, c % 8)) = v;
+        for (int k = 0; k < CH; ++k) {
+          const int idx = k * 32 + lane, row = idx / CH, c = half * CH + idx % CH;
+          const int tok = __shfl_sync(0xffffffffu, token, row);
+          const bool valid = __shfl_sync(0xffffffffu, row_valid ? 1 : 0, row) != 0;
+          v[k] = make_uint4(0, 0, 0, 0);
+          if (valid) v[k] = __ldg(reinterpret_cast<const uint4*>(p.q + (static_cast<size_t>(tok) * p.n_heads + w.head) * D) + c);
+        }
+#pragma unroll
+        for (int k = 0; k < CH; ++k) {
+          const int idx = k * 32 + lane, row = idx / CH, c = half * CH + idx % CH;
+          *reinterpret_cast<uint4*>(sq + (c / 8) * SM::BLOCK_BYTES + sw128_offset((r & ~31) + row, c % 8)) = v[k];
         }
         fence_proxy_async_smem();
         tc_fence_before_sync();  // orders this thread's TMEM reads of the previous item before the arrive
@@ -461,31 +471,93 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const __grid_cons
       tc_fence_after_sync();
       const float inv = (l_sum > 0.f) ? 1.f / l_sum : 0.f;
       const float mult = (w.out_mode == OUT_PARTIAL) ? 1.f : inv;
-      const size_t row_elem = (static_cast<size_t>(token) * p.n_heads + w.head) * D + half * OC;
-#pragma unroll 1
-      for (int ch = 0; ch < OC / 32; ++ch) {
-        uint32_t v[32];
-        tmem_ld32(o_addr + ch * 32, v);
-        tmem_wait_ld();
-        if (!row_valid) continue;
+      if constexpr (D == 128) {
+        // The thread holds its row's OC output columns, but one row per lane is the worst pattern for global stores
+        // (32 lines per instruction: 4096 line visits per tile, 4-5 us per item).  So the warp turns its 32 x OC block
+        // through shared memory - its 4 KB of this tile's query buffer, which the last S product has finished reading
+        // (the O product committed to bar_o_full was issued after it) - and stores whole 128-byte lines: 8 lanes a row.
+        uint8_t* stg = sq + (half * 4 + (warp & 3)) * 4096;
+        const int row0 = r & ~31;  // first row of this warp inside the tile
         if (w.out_mode == OUT_BF16) {
-          uint4* dst = reinterpret_cast<uint4*>(p.out + row_elem + ch * 32);
-#pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            uint4 o4;
-            o4.x = pack_bf16x2(__uint_as_float(v[8 * i + 0]) * mult, __uint_as_float(v[8 * i + 1]) * mult);
-            o4.y = pack_bf16x2(__uint_as_float(v[8 * i + 2]) * mult, __uint_as_float(v[8 * i + 3]) * mult);
-            o4.z = pack_bf16x2(__uint_as_float(v[8 * i + 4]) * mult, __uint_as_float(v[8 * i + 5]) * mult);
-            o4.w = pack_bf16x2(__uint_as_float(v[8 * i + 6]) * mult, __uint_as_float(v[8 * i + 7]) * mult);
-            dst[i] = o4;
+          constexpr int U = OC / 8;  // 16-byte units of a row's half: 8 (d = 128) or 4 (d = 64)
+  #pragma unroll 1
+          for (int ch = 0; ch < OC / 32; ++ch) {
+            uint32_t v[32];
+            tmem_ld32(o_addr + ch * 32, v);
+            tmem_wait_ld();
+  #pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              uint4 o4;
+              o4.x = pack_bf16x2(__uint_as_float(v[8 * i + 0]) * mult, __uint_as_float(v[8 * i + 1]) * mult);
+              o4.y = pack_bf16x2(__uint_as_float(v[8 * i + 2]) * mult, __uint_as_float(v[8 * i + 3]) * mult);
+              o4.z = pack_bf16x2(__uint_as_float(v[8 * i + 4]) * mult, __uint_as_float(v[8 * i + 5]) * mult);
+              o4.w = pack_bf16x2(__uint_as_float(v[8 * i + 6]) * mult, __uint_as_float(v[8 * i + 7]) * mult);
+              *reinterpret_cast<uint4*>(stg + lane * 128 + (((ch * 4 + i) ^ (lane & 7)) << 4)) = o4;
+            }
           }
+          __syncwarp();
+  #pragma unroll
+          for (int k = 0; k < U; ++k) {
+            const int idx = k * 32 + lane, row = idx / U, u = idx % U;
+            const uint4 val = *reinterpret_cast<const uint4*>(stg + row * 128 + ((u ^ (row & 7)) << 4));
+            const int tok = __shfl_sync(0xffffffffu, token, row);
+            const bool valid = __shfl_sync(0xffffffffu, row_valid ? 1 : 0, row) != 0;
+            if (valid)
+              *reinterpret_cast<uint4*>(p.out + (static_cast<size_t>(tok) * p.n_heads + w.head) * D + half * OC + u * 8) = val;
+          }
+          __syncwarp();
         } else {
-          float* base = p.part_o + (static_cast<size_t>(w.out_slot) * 256 + t * 128 + r) * D + half * OC;
-          float4* dst = reinterpret_cast<float4*>(base + ch * 32);
+          float* base = p.part_o + (static_cast<size_t>(w.out_slot) * 256 + t * 128 + row0) * D + half * OC;
+  #pragma unroll 1
+          for (int ch = 0; ch < OC / 32; ++ch) {
+            uint32_t v[32];
+            tmem_ld32(o_addr + ch * 32, v);
+            tmem_wait_ld();
+  #pragma unroll
+            for (int i = 0; i < 8; ++i)
+              *reinterpret_cast<float4*>(stg + lane * 128 + ((i ^ (lane & 7)) << 4)) =
+                  make_float4(__uint_as_float(v[4 * i + 0]) * mult, __uint_as_float(v[4 * i + 1]) * mult,
+                              __uint_as_float(v[4 * i + 2]) * mult, __uint_as_float(v[4 * i + 3]) * mult);
+            __syncwarp();
+  #pragma unroll
+            for (int k = 0; k < 8; ++k) {
+              const int idx = k * 32 + lane, row = idx >> 3, u = idx & 7;
+              const float4 val = *reinterpret_cast<const float4*>(stg + row * 128 + ((u ^ (row & 7)) << 4));
+              const bool valid = __shfl_sync(0xffffffffu, row_valid ? 1 : 0, row) != 0;
+              if (valid) *reinterpret_cast<float4*>(base + static_cast<size_t>(row) * D + ch * 32 + u * 4) = val;
+            }
+            __syncwarp();
+          }
+        }
+      } else
+      {
+        // head_dim 64: a tile's query buffer (16 KB) is too small to turn the fp32 block through; one row per lane
+        const size_t row_elem = (static_cast<size_t>(token) * p.n_heads + w.head) * D + half * OC;
+#pragma unroll 1
+        for (int ch = 0; ch < OC / 32; ++ch) {
+          uint32_t v[32];
+          tmem_ld32(o_addr + ch * 32, v);
+          tmem_wait_ld();
+          if (!row_valid) continue;
+          if (w.out_mode == OUT_BF16) {
+            uint4* dst = reinterpret_cast<uint4*>(p.out + row_elem + ch * 32);
 #pragma unroll
-          for (int i = 0; i < 8; ++i)
-            dst[i] = make_float4(__uint_as_float(v[4 * i + 0]) * mult, __uint_as_float(v[4 * i + 1]) * mult,
-                                 __uint_as_float(v[4 * i + 2]) * mult, __uint_as_float(v[4 * i + 3]) * mult);
+            for (int i = 0; i < 4; ++i) {
+              uint4 o4;
+              o4.x = pack_bf16x2(__uint_as_float(v[8 * i + 0]) * mult, __uint_as_float(v[8 * i + 1]) * mult);
+              o4.y = pack_bf16x2(__uint_as_float(v[8 * i + 2]) * mult, __uint_as_float(v[8 * i + 3]) * mult);
+              o4.z = pack_bf16x2(__uint_as_float(v[8 * i + 4]) * mult, __uint_as_float(v[8 * i + 5]) * mult);
+              o4.w = pack_bf16x2(__uint_as_float(v[8 * i + 6]) * mult, __uint_as_float(v[8 * i + 7]) * mult);
+              dst[i] = o4;
+            }
+          } else {
+            float* base = p.part_o + (static_cast<size_t>(w.out_slot) * 256 + t * 128 + r) * D + half * OC;
+            float4* dst = reinterpret_cast<float4*>(base + ch * 32);
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+              dst[i] = make_float4(__uint_as_float(v[4 * i + 0]) * mult, __uint_as_float(v[4 * i + 1]) * mult,
+                                   __uint_as_float(v[4 * i + 2]) * mult, __uint_as_float(v[4 * i + 3]) * mult);
+          }
         }
       }
       if (row_valid && half == 0 && w.out_mode == OUT_PARTIAL) {
