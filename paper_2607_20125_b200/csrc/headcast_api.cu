@@ -251,15 +251,30 @@ WorkItem range_item(int head, int map, int x0, long long row0, int n_keys) {
   return w;
 }
 
-// Cost model of the scheduler, in units of the time one key tile takes with both query tiles in flight
-// (fitted to per-item timings from headcast_read_trace on B200): a lone query tile still needs 0.82 of that
-// because the chain S -> softmax -> P -> next S is latency bound; every item pays for its query load, pipeline
-// fill and epilogue; a partial result costs an extra round trip through global memory; the tiles of Spatial items
-// measure 5 % slower and the CTAs that hold nothing else finished last, hence the factor on them.
-constexpr double TILE_COST_PAIR = 1.0, TILE_COST_SINGLE = 0.82;
-constexpr double ITEM_OVERHEAD = 3.5, ITEM_OVERHEAD_SINGLE = 2.5;
-constexpr double PARTIAL_EXTRA = 1.0;
-constexpr double SPATIAL_FACTOR = 1.10;  // tiles of Spatial items (queries gathered by cell, short cell-major key runs) take longer
+// Cost model of the scheduler, in units of the time one key tile takes with both query tiles in flight (about 2.0 us),
+// fitted by least squares to the per-item timings of headcast_read_trace on B200 (480P, 720P and 1080P work lists,
+// residual 1-3 % of an item): a lone query tile still needs 0.86 of that because the chain S -> softmax -> P -> next S
+// is latency bound; every item pays for its query load, pipeline fill and epilogue; a partial result costs an extra
+// round trip through global memory; the tiles of Spatial items measure 2 % slower.
+#ifndef HC_COST_ITEM
+#define HC_COST_ITEM 2.4
+#endif
+#ifndef HC_COST_ITEM_SINGLE
+#define HC_COST_ITEM_SINGLE 1.0
+#endif
+#ifndef HC_COST_PARTIAL
+#define HC_COST_PARTIAL 0.75
+#endif
+#ifndef HC_COST_SPATIAL
+#define HC_COST_SPATIAL 1.02
+#endif
+#ifndef HC_COST_SINGLE
+#define HC_COST_SINGLE 0.86
+#endif
+constexpr double TILE_COST_PAIR = 1.0, TILE_COST_SINGLE = HC_COST_SINGLE;
+constexpr double ITEM_OVERHEAD = HC_COST_ITEM, ITEM_OVERHEAD_SINGLE = HC_COST_ITEM_SINGLE;
+constexpr double PARTIAL_EXTRA = HC_COST_PARTIAL;
+constexpr double SPATIAL_FACTOR = HC_COST_SPATIAL;  // tiles of Spatial items (queries gathered by cell, short cell-major key runs)
 constexpr int MIN_PART_TILES = 4;  // never cut a key range into pieces shorter than this
 
 double tile_cost(const WorkItem& w) {

@@ -95,11 +95,11 @@ def check_plan(w, labels, n_filled, n_ctas, dense=False):
             want_tiles[h] = -(-(n_filled * w.frames_per_block * sizes[cell]) // 128)
     assert np.array_equal(covered, want_tiles)
     assert np.all(finals <= 1)
-    # load balance under the scheduler's own cost model: per key tile 1 (query pair) or 0.82 (lone query tile), times
-    # 1.1 for Spatial items; per item 3.5 or 2.5, +1 per partial result
+    # load balance under the scheduler's own cost model: per key tile 1 (query pair) or 0.86 (lone query tile), times
+    # 1.02 for Spatial items; per item 2.4 or 1.0, +0.75 per partial result
     pair = items[:, F["q_count1"]] > 0
-    cost = np.where(pair, 1.0, 0.82) * np.where(items[:, F["cell"]] >= 0, 1.1, 1.0) \
-        * (items[:, F["tile_end"]] - items[:, F["tile_begin"]]) + np.where(pair, 3.5, 2.5) + (items[:, F["out_mode"]] == 1)
+    cost = np.where(pair, 1.0, 0.86) * np.where(items[:, F["cell"]] >= 0, 1.02, 1.0) \
+        * (items[:, F["tile_end"]] - items[:, F["tile_begin"]]) + np.where(pair, 2.4, 1.0) + 0.75 * (items[:, F["out_mode"]] == 1)
     per_cta = np.array([cost[first[b]:first[b + 1]].sum() for b in range(n_ctas)])
     return items, per_cta
 
