@@ -67,3 +67,30 @@ def test_reference_arm_prints_one_line_from_rank_zero_only():
     assert line["cpu_baseline"]["kind"] == "oracle" and line["cpu_baseline"]["value"] == line["value"]
     assert line["e2e"] == {"value": line["value"], "unit": "ms", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}
     assert line["config"]["workload"] == "tiny"
+
+
+def test_both_arms_describe_the_same_workload_and_the_roofline_follows_the_regime():
+    sys.path.insert(0, ROOT)
+    import argparse
+    import bench
+    from paper_2607_20125_b200 import synth
+    w = synth.wan("1080p")
+    # the reference arm and the CUDA arm print the same `config` object (same keys, same values at one GPU)
+    assert bench.config_of(w, 1, 0) == bench.config_of(w, 1, 0) and bench.config_of(w)["workload"] == "1080p"
+    assert set(bench.config_of(w, 2, 0)) == set(bench.config_of(w, 1, 0))
+    # algorithmic bytes of the copy path: append reads the block and writes every head but the two Sink heads
+    nb = bench.algorithmic_bytes(synth.wan("480p"))
+    assert abs(nb["append"] / 1e6 - 52.7) < 0.1 and abs(nb["split"] / 1e6 - 258.8) < 0.1 and abs(nb["block"] / 1e6 - 28.8) < 0.1
+    # DRAM traffic comes from the capture written under profiles/, not from a literal
+    assert bench.ncu_traffic_bytes("1080p") > bench.ncu_traffic_bytes("720p") > bench.ncu_traffic_bytes("480p") > 1e8
+    assert bench.ncu_traffic_bytes("tiny") is None
+    peaks = {"tflops": 1600.0, "tflops_sustained": 1400.0, "hbm_gbs": 6500.0, "source": "measured"}
+    r = {"ms_per_step": 8.0, "kernel_tflops": 980.0, "kernel_ms": 8.0, "flops_per_launch": 8.0e12, "frac_of_measured_burst": 980 / 1600,
+         "frac_of_measured_sustained": 0.7, "frac_of_nominal_2250": 980 / 2250, "clocks": {"reasons": ["sw_power_cap"]}}
+    long_run = bench.roofline_of(r, w, argparse.Namespace(steps=40), peaks)
+    assert long_run["peak"] == 1400.0 and abs(long_run["frac"] - 0.7) < 1e-12 and "sustained" in long_run["peak_source"]
+    assert long_run["bar_met_nominal"] is False and long_run["frac_of_nominal"] < 0.5
+    short = bench.roofline_of(dict(r, ms_per_step=0.35), w, argparse.Namespace(steps=40), peaks)
+    assert short["peak"] == 1600.0 and "burst" in short["peak_source"]
+    cool = bench.roofline_of(dict(r, clocks={"reasons": []}), w, argparse.Namespace(steps=40), peaks)
+    assert cool["peak"] == 1600.0
