@@ -86,11 +86,15 @@ def test_both_arms_describe_the_same_workload_and_the_roofline_follows_the_regim
     assert bench.ncu_traffic_bytes("tiny") is None
     peaks = {"tflops": 1600.0, "tflops_sustained": 1400.0, "hbm_gbs": 6500.0, "source": "measured"}
     r = {"ms_per_step": 8.0, "kernel_tflops": 980.0, "kernel_ms": 8.0, "flops_per_launch": 8.0e12, "frac_of_measured_burst": 980 / 1600,
-         "frac_of_measured_sustained": 0.7, "frac_of_nominal_2250": 980 / 2250, "clocks": {"reasons": ["sw_power_cap"]}}
+         "frac_of_measured_sustained": 0.7, "frac_of_nominal_2250": 980 / 2250,
+         "clocks": {"reasons": ["sw_power_cap"], "sm_mhz": 1650.0, "sm_max_mhz": 1965}}
     long_run = bench.roofline_of(r, w, argparse.Namespace(steps=40), peaks)
     assert long_run["peak"] == 1400.0 and abs(long_run["frac"] - 0.7) < 1e-12 and "sustained" in long_run["peak_source"]
     assert long_run["bar_met_nominal"] is False and long_run["frac_of_nominal"] < 0.5
     short = bench.roofline_of(dict(r, ms_per_step=0.35), w, argparse.Namespace(steps=40), peaks)
-    assert short["peak"] == 1600.0 and "burst" in short["peak_source"]
-    cool = bench.roofline_of(dict(r, clocks={"reasons": []}), w, argparse.Namespace(steps=40), peaks)
+    assert short["peak"] == 1600.0 and "burst" in short["peak_source"]  # 14 ms of steps: a burst
+    cool = bench.roofline_of(dict(r, clocks={"reasons": [], "sm_mhz": 1965.0, "sm_max_mhz": 1965}), w, argparse.Namespace(steps=40), peaks)
     assert cool["peak"] == 1600.0
+    fast = bench.roofline_of(dict(r, clocks={"reasons": ["sw_power_cap"], "sm_mhz": 1900.0, "sm_max_mhz": 1965}), w,
+                             argparse.Namespace(steps=40), peaks)
+    assert fast["peak"] == 1600.0  # the cap touched, the clock not held down: still the burst figure
