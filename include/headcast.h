@@ -190,7 +190,8 @@ int headcast_last_attention_kernel_ms(headcast_ctx* ctx, float* ms_host);
 /* Scheduling aid.  With enable != 0 every later attention launch records, per work item, the GPU global timer
  * (ns) at which the item's first query tile started and finished.  headcast_read_trace synchronises the device
  * and writes, for each work item of the most recent attention launch, 8 int64 values to rows_host
- * ([capacity][8]): CTA index, head, Spatial cell (-1 if none), query rows, key tiles, output mode
+ * ([capacity][8]): CTA index (the CTA count for items of the shared queue), head, Spatial cell (-1 if none), query
+ * rows, key tiles, output mode
  * (0 final, 1 partial, 2 fp32), start ns, end ns.  *n_items_host receives the item count. */
 int headcast_set_tracing(headcast_ctx* ctx, int32_t enable);
 int headcast_read_trace(headcast_ctx* ctx, int64_t* rows_host, int32_t capacity, int32_t* n_items_host);
@@ -201,7 +202,9 @@ int headcast_read_trace(headcast_ctx* ctx, int64_t* rows_host, int32_t capacity,
  * tile 0 and 1, buffer (0 monolithic, 1 Sink-Dummy, 2 Global, 3 Spatial), element column, first key row, row stride
  * between key segments, keys per segment, 128-key tiles per segment, first and one-past-last tile of this item,
  * output mode (0 final, 1 partial to be merged), partial slot.  items_host has room for `capacity` items,
- * cta_first_host for n_ctas + 1 entries (items of CTA b are [cta_first[b], cta_first[b+1])); either may be NULL. */
+ * cta_first_host for n_ctas + 1 entries (items of CTA b are [cta_first[b], cta_first[b+1])); either may be NULL.
+ * Items from cta_first[n_ctas] up to *n_items_host belong to no CTA: they form the shared queue (the last ~2 % of
+ * the work, cut into small pieces) that CTAs draw from, in order, once their own lists are done. */
 int headcast_plan_schedule(const headcast_config* cfg, const int32_t* labels_host, int32_t n_filled, int32_t n_ctas,
                            int32_t dense, int32_t* items_host, int32_t capacity, int32_t* n_items_host,
                            int32_t* cta_first_host);

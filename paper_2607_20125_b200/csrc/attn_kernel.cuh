@@ -57,6 +57,10 @@ struct AttnParams {
   int32_t n_heads, tokens_per_frame, grid_w, block_tokens;
   float scale_log2e;       // softmax scale * log2(e)
   int32_t* status;
+  // dynamic tail: when a CTA has finished its own list it draws items [dyn_first, dyn_end) of `items` from a shared
+  // queue; dyn_counter[0] is the next queue position, dyn_counter[1] counts CTAs that are done (the last clears both)
+  int32_t dyn_first, dyn_end;
+  int32_t* dyn_counter;
   unsigned long long* trace;  // optional [2 * n_items]: globaltimer (ns) when query tile 0's warpgroup starts / ends an item
   // Spatial proxy only
   int32_t radius;
@@ -147,6 +151,8 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const __grid_cons
   __shared__ uint64_t bar_kv_full[KV_SLOTS], bar_kv_free[KV_SLOTS];
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag;
+  __shared__ uint64_t bar_dyn[4];
+  __shared__ int32_t dyn_item[4];
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   if (tid == 0) {
@@ -163,6 +169,7 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const __grid_cons
       mbar_init(&bar_kv_full[s], 1);
       mbar_init(&bar_kv_free[s], 1);
     }
+    for (int s = 0; s < 4; ++s) mbar_init(&bar_dyn[s], 1);
     abort_flag = 0;
     fence_mbar_init();
   }
@@ -177,6 +184,42 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const __grid_cons
   volatile int* abortp = &abort_flag;
 
   const int item_lo = p.cta_first[blockIdx.x], item_hi = p.cta_first[blockIdx.x + 1];
+  const bool has_queue = p.dyn_end > p.dyn_first;
+  // Items come from the CTA's own list first, then from the shared queue.  The producer thread draws the queue
+  // position and publishes it through a ring of four shared-memory slots; it runs at most two key tiles (less than
+  // one item) ahead of the other roles, so a slot is read long before its fourth successor is written.
+  struct ItemCursor { int it; bool in_queue; uint32_t k; };
+  // issuer and softmax warps: advance to the next item (false: no more)
+  auto next_item = [&](ItemCursor& cur) -> bool {
+    if (!cur.in_queue) {
+      if (cur.it + 1 < item_hi) { ++cur.it; return true; }
+      cur.in_queue = true;
+    }
+    if (!has_queue) return false;
+    if (!mbar_wait(&bar_dyn[cur.k & 3], (cur.k >> 2) & 1, abortp, p.status, 51)) return false;
+    cur.it = dyn_item[cur.k & 3];
+    ++cur.k;
+    return cur.it >= 0;
+  };
+  // producer thread: the same, but it is the one that draws from the queue and tells the others
+  auto next_item_producer = [&](ItemCursor& cur) -> bool {
+    if (!cur.in_queue) {
+      if (cur.it + 1 < item_hi) { ++cur.it; return true; }
+      cur.in_queue = true;
+    }
+    if (!has_queue) return false;
+    const int pos = atomicAdd(&p.dyn_counter[0], 1);
+    const int v = (pos < p.dyn_end - p.dyn_first) ? p.dyn_first + pos : -1;
+    dyn_item[cur.k & 3] = v;
+    mbar_arrive(&bar_dyn[cur.k & 3]);  // release: the slot is written before the arrival is seen
+    ++cur.k;
+    cur.it = v;
+    if (v < 0 && atomicAdd(&p.dyn_counter[1], 1) == static_cast<int>(gridDim.x) - 1) {
+      p.dyn_counter[0] = 0;  // every CTA has drawn its end marker: the queue is ready for the next launch
+      p.dyn_counter[1] = 0;
+    }
+    return v >= 0;
+  };
 
 
   if (warp == 0) {
@@ -192,7 +235,9 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const __grid_cons
 #else
       const uint64_t pol_keep = l2_policy_evict_normal();
 #endif
-      for (int it = item_lo; it < item_hi && ok; ++it) {
+      ItemCursor cur = {item_lo - 1, false, 0u};
+      while (ok && next_item_producer(cur)) {
+        const int it = cur.it;
         const WorkItem w = p.items[it];
         const CUtensorMap* kmap = &p.maps[2 * w.kv_map];
         const CUtensorMap* vmap = kmap + 1;
@@ -239,7 +284,9 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const __grid_cons
         mma_block_ts8(tmem + O_COL + t * 128, tmem + S_COL + t * 128, v_desc + ((st * SM::TILE_BYTES) >> 4), idesc_o,
                       accumulate ? 1u : 0u);
       };
-      for (int it = item_lo; it < item_hi && ok; ++it) {
+      ItemCursor cur = {item_lo - 1, false, 0u};
+      while (ok && next_item(cur)) {
+        const int it = cur.it;
         const WorkItem w = p.items[it];
         const int nt = w.tile_end - w.tile_begin;
         const int n_q = w.q_count[1] > 0 ? 2 : 1;
@@ -310,7 +357,9 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const __grid_cons
       theirs = pair_val[t][par][half ^ 1][r];
       return true;
     };
-    for (int it = item_lo; it < item_hi && ok; ++it) {
+    ItemCursor cur = {item_lo - 1, false, 0u};
+    while (ok && next_item(cur)) {
+      const int it = cur.it;
       const WorkItem w = p.items[it];
       if (w.q_count[t] == 0) continue;
       if (p.trace && t == 0 && r == 0 && half == 0) p.trace[2 * it] = global_timer_ns();

@@ -59,6 +59,7 @@ struct Schedule {
   DevBuf<ClsGroup> cls_groups_dev;
   DevBuf<ClsPart> cls_parts_dev;
   int n_slots = 0;
+  int dyn_first = 0, dyn_end = 0;  // items [dyn_first, dyn_end) form the shared queue the CTAs draw from when their own list is done
   bool uploaded = false;
   double flops = 0.0;
   void release() {
@@ -107,6 +108,7 @@ struct headcast_ctx {
   MoveMaps move_recent[8];
   int move_next = 0;
   int32_t* status_dev = nullptr;
+  int32_t* dyn_counter_dev = nullptr;  // [2]: next queue position, CTAs done (the last one clears both)
 
   Schedule sched_dense, sched_hc, sched_cls, sched_proxy;
   // headcast_attend_host: the stages of its pipeline, each with its own work list - the first half of the Global
@@ -297,7 +299,9 @@ void finalize_schedule(headcast_ctx* c, Schedule& s, std::vector<Proto>& protos,
   s.combine.clear();
   s.n_slots = 0;
   const int n_cta = c->n_sm;
-  std::vector<std::vector<WorkItem>> bins(n_cta);
+  std::vector<std::vector<WorkItem>> bins(n_cta + 1);  // bins[n_cta]: the shared queue (dynamic tail)
+  bool tail_mode = false;
+  int tail_piece_tiles = 8;
   std::stable_sort(protos.begin(), protos.end(),
                    [](const Proto& a, const Proto& b) { return item_cost(a.w) > item_cost(b.w); });
   if (allow_split) {
@@ -312,13 +316,15 @@ void finalize_schedule(headcast_ctx* c, Schedule& s, std::vector<Proto>& protos,
     int slot_base = 0;
     auto lay_out = [&](double quota) -> double {
       for (int b = 0; b < n_cta; ++b) bins[b].resize(bin_base[b]);
+      bins[n_cta].clear();
       s.combine.resize(combine_base);
       cls_raw.resize(cls_base);
       s.n_slots = slot_base;
       int cta = 0;
       double room = quota, last_load = 0.0;
+      const int last_bin = tail_mode ? n_cta : n_cta - 1;
       auto next_cta = [&]() {
-        if (cta + 1 < n_cta) {
+        if (cta < last_bin) {
           ++cta;
           room = quota;
         }
@@ -332,7 +338,11 @@ void finalize_schedule(headcast_ctx* c, Schedule& s, std::vector<Proto>& protos,
           const int left = p.n_tiles - begin;
           const double need = per_tile * left + overhead + (begin > 0 ? PARTIAL_EXTRA : 0.0);
           int take = left;
-          if (need > room && cta + 1 < n_cta) {
+          if (tail_mode && cta == n_cta) {
+            // the shared queue: pieces of a fixed size, drawn by whichever CTA is free
+            take = std::min(left, tail_piece_tiles);
+            if (left - take < MIN_PART_TILES) take = left;
+          } else if (need > room && cta < last_bin) {
             // as many tiles as fit, but both pieces must be worth having
             const int can = std::min(static_cast<int>(std::floor((room - overhead - PARTIAL_EXTRA) / per_tile)),
                                      left - MIN_PART_TILES);
@@ -384,6 +394,7 @@ void finalize_schedule(headcast_ctx* c, Schedule& s, std::vector<Proto>& protos,
       for (int b = 0; b < n_cta; ++b) n += bins[b].size() == bin_base[b];
       return n;
     };
+    double tail_budget = 0.0;
     auto place = [&](size_t first, size_t last) {  // spreads protos [first, last) over all CTAs, after what is there
       first_proto = first;
       last_proto = last;
@@ -393,6 +404,16 @@ void finalize_schedule(headcast_ctx* c, Schedule& s, std::vector<Proto>& protos,
         biggest = std::max(biggest, item_cost(protos[pi].w));
       }
       const double ideal = total / n_cta;
+      if (tail_budget > 0.0 && last == protos.size() && total > 20.0 * n_cta) {
+        // last phase: every CTA gets an equal share of all but the tail budget; the rest goes to the shared queue
+        const double budget = std::min(tail_budget, 0.5 * total);
+        tail_mode = true;
+        tail_piece_tiles = std::max(8, static_cast<int>(budget / (4.0 * n_cta)));
+        lay_out((total - budget) / n_cta);
+        tail_mode = false;
+        for (int b = 0; b < n_cta; ++b) bin_base[b] = bins[b].size();
+        return;
+      }
       double lo = ideal, hi = ideal + biggest + ITEM_OVERHEAD + PARTIAL_EXTRA;
       while (!fits(hi)) hi *= 1.25;
       for (int iter = 0; iter < 24 && hi - lo > 0.25; ++iter) {
@@ -461,6 +482,14 @@ void finalize_schedule(headcast_ctx* c, Schedule& s, std::vector<Proto>& protos,
         }
         it->cost += item_cost(p.w);
       }
+      // Dynamic tail.  Identical work takes +-3 % longer or shorter from SM to SM, which no static list can absorb: the
+      // last HC_TAIL_FRAC of the launch's work is held back from the equal shares and cut into small pieces that the
+      // CTAs draw from a shared queue when their own lists are done (measured: 0.02 is the best of 0.02 / 0.04 / 0.06;
+      // -3.5 % at 480P, -0.7 % at 720P, -0.5 % at 1080P).  Not for classification sweeps (their pieces are merged by group).
+#ifndef HC_TAIL_FRAC
+#define HC_TAIL_FRAC 0.02
+#endif
+      if (s.cls_groups.empty() && all_cost > 40.0 * n_cta) tail_budget = HC_TAIL_FRAC * all_cost;
       std::stable_sort(streams.begin(), streams.end(), [](const Stream& a, const Stream& b) { return a.cost > b.cost; });
       // first-fit of the streams into phases; a phase too light to be cut 148 ways is dissolved again
       std::vector<double> phase_cost;
@@ -521,6 +550,17 @@ void finalize_schedule(headcast_ctx* c, Schedule& s, std::vector<Proto>& protos,
           }
         }
         protos.swap(expanded);
+        // what belongs to no phase (short streams, Spatial cells, phases too light to be cut 148 ways) goes FIRST, the
+        // phases follow: the launch then ends inside a long stream, whose last stretch feeds the shared queue
+        auto heavy = [&](const Proto& p) { return p.phase >= 0 && phase_cost[p.phase] >= 60.0 * n_cta; };
+        bool any_heavy = false;
+        for (const Proto& p : protos) any_heavy = any_heavy || heavy(p);
+        if (any_heavy) {
+          auto mid0 = std::stable_partition(protos.begin(), protos.end(), [&](const Proto& p) { return !heavy(p); });
+          const size_t n_left = static_cast<size_t>(mid0 - protos.begin());
+          if (n_left > 0) place(0, n_left);
+          done = n_left;
+        }
         for (size_t ph = 0; ph < phase_cost.size(); ++ph) {
           if (phase_cost[ph] < 60.0 * n_cta) continue;
           auto in_phase = [&](const Proto& p) { return p.phase == static_cast<int>(ph); };
@@ -537,7 +577,7 @@ void finalize_schedule(headcast_ctx* c, Schedule& s, std::vector<Proto>& protos,
     if (s.cls_groups.empty()) {
       struct Piece { int bin, pos, tile_begin; };
       std::vector<std::vector<Piece>> by_group;
-      for (int b = 0; b < n_cta; ++b)
+      for (int b = 0; b <= n_cta; ++b)
         for (size_t i = 0; i < bins[b].size(); ++i) {
           const WorkItem& w = bins[b][i];
           if (static_cast<size_t>(w.out_slot) >= by_group.size()) by_group.resize(w.out_slot + 1);
@@ -598,6 +638,9 @@ void finalize_schedule(headcast_ctx* c, Schedule& s, std::vector<Proto>& protos,
     s.items.insert(s.items.end(), bins[b].begin(), bins[b].end());
   }
   s.cta_first[n_cta] = static_cast<int32_t>(s.items.size());
+  s.dyn_first = static_cast<int32_t>(s.items.size());
+  s.items.insert(s.items.end(), bins[n_cta].begin(), bins[n_cta].end());
+  s.dyn_end = static_cast<int32_t>(s.items.size());
   s.uploaded = false;
 }
 
@@ -734,6 +777,9 @@ int run_schedule(headcast_ctx* c, Schedule& s, const void* q, void* out, bool pr
   p.block_tokens = c->L;
   p.scale_log2e = c->scale * 1.4426950408889634f;
   p.status = c->status_dev;
+  p.dyn_first = s.dyn_first;
+  p.dyn_end = s.dyn_end;
+  p.dyn_counter = c->dyn_counter_dev;
   p.trace = nullptr;
   if (c->tracing) {
     const size_t trace_words = 2 * s.items.size();
@@ -980,6 +1026,7 @@ int read_status(headcast_ctx* c, cudaStream_t st) {
   HC_CUDA(c, cudaStreamSynchronize(st));
   if (status != 0) {
     cudaMemsetAsync(c->status_dev, 0, sizeof(int32_t), st);
+    cudaMemsetAsync(c->dyn_counter_dev, 0, 2 * sizeof(int32_t), st);  // a kernel that gave up may have left the queue half drawn
     return fail(c, HC_ERR_TIMEOUT, "a kernel gave up on a bounded wait (site %d)", status);
   }
   return HC_OK;
@@ -1145,6 +1192,8 @@ int headcast_create(const headcast_config* cfg, headcast_ctx** out) {
   step(cudaMalloc(&c->sp_nc, c->T_f * sizeof(int32_t)));
   step(cudaMalloc(&c->cells_dev, c->cells.size() * sizeof(CellGeom)));
   step(cudaMalloc(&c->status_dev, sizeof(int32_t)));
+  step(cudaMalloc(&c->dyn_counter_dev, 2 * sizeof(int32_t)));
+  if (e == cudaSuccess) step(cudaMemset(c->dyn_counter_dev, 0, 2 * sizeof(int32_t)));
   if (c->move_ok) step(cudaMalloc(&c->move_boxes_dev, std::max<size_t>(1, c->move_boxes.size()) * sizeof(MoveBox)));
   if (e == cudaSuccess) {
     step(cudaMemset(c->mono_k, 0, mono_bytes));
@@ -1180,7 +1229,7 @@ int headcast_destroy(headcast_ctx* c) {
   if (c->mono_k) cudaFreeAsync(c->mono_k, nullptr);
   if (c->mono_v) cudaFreeAsync(c->mono_v, nullptr);
   cudaDeviceSynchronize();
-  void* ptrs[] = {c->arena_k, c->arena_v, c->sp_base, c->sp_nc, c->cells_dev, c->status_dev, c->move_boxes_dev};
+  void* ptrs[] = {c->arena_k, c->arena_v, c->sp_base, c->sp_nc, c->cells_dev, c->status_dev, c->dyn_counter_dev, c->move_boxes_dev};
   for (void* p : ptrs)
     if (p) cudaFree(p);
   if (c->ev_a) cudaEventDestroy(c->ev_a);

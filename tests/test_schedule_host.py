@@ -38,7 +38,7 @@ def check_plan(w, labels, n_filled, n_ctas, dense=False):
               geom.col_edges[j + 1] - geom.col_edges[j])
              for i in range(len(geom.row_edges) - 1) for j in range(len(geom.col_edges) - 1)]
     L, H = geom.block_tokens, w.n_heads
-    assert first[0] == 0 and first[-1] == len(items) and np.all(np.diff(first) >= 0)
+    assert first[0] == 0 and first[-1] <= len(items) and np.all(np.diff(first) >= 0)
     covered = np.zeros((H, L), dtype=np.int64)   # key tiles seen by every (head, row)
     finals = np.zeros((H, L), dtype=np.int64)
     groups = {}
@@ -101,6 +101,14 @@ def check_plan(w, labels, n_filled, n_ctas, dense=False):
     cost = np.where(pair, 1.0, 0.86) * np.where(items[:, F["cell"]] >= 0, 1.02, 1.0) \
         * (items[:, F["tile_end"]] - items[:, F["tile_begin"]]) + np.where(pair, 2.4, 1.0) + 0.75 * (items[:, F["out_mode"]] == 1)
     per_cta = np.array([cost[first[b]:first[b + 1]].sum() for b in range(n_ctas)])
+    # what lies after the last CTA's list is the shared queue that CTAs draw from once their own lists are done: a
+    # small part of the launch, in pieces small enough that the last one drawn cannot delay the end by much
+    queue = cost[first[-1]:]
+    if queue.size:
+        # (2 % of the launch by design, plus the cost of the cuts that the equal static shares did not allow for)
+        assert queue.sum() <= 0.08 * cost.sum() + 40.0
+        q_tiles = (items[first[-1]:, F["tile_end"]] - items[first[-1]:, F["tile_begin"]]).max()
+        assert q_tiles <= max(8, 0.02 * cost.sum() / (4 * n_ctas)) + 4  # a piece, plus a remainder too short to stand alone
     return items, per_cta
 
 
@@ -128,6 +136,10 @@ def test_long_key_streams_are_swept_chunk_by_chunk_by_all_ctas():
         bounds = [total_tiles * k // n_chunks for k in range(n_chunks + 1)]
         chunk_of = lambda it: next(k for k in range(n_chunks) if bounds[k] <= it[F["tile_begin"]] < bounds[k + 1])
         busy = 0
+        for it in items[first[-1]:]:  # pieces in the shared queue keep to the chunk boundaries too
+            if it[F["head"]] == h:
+                k = chunk_of(it)
+                assert bounds[k] <= it[F["tile_begin"]] < it[F["tile_end"]] <= bounds[k + 1]
         for b in range(148):
             seq = [chunk_of(it) for it in items[first[b]:first[b + 1]] if it[F["head"]] == h]
             for it in items[first[b]:first[b + 1]]:
