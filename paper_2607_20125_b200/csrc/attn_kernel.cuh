@@ -636,6 +636,14 @@ struct CombineEntry {
 
 constexpr int COMBINE_ROWS = 16;  // query rows per block of combine_kernel
 
+// Streaming 16-byte load, as a volatile statement: the compiler keeps such loads in program order, so a batch written
+// before its first use really is in flight together (left to itself it sinks each load to its use to save registers).
+__device__ __forceinline__ float4 ld_stream_f4(const float4* p) {
+  float4 v;
+  asm volatile("ld.global.cs.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p));
+  return v;
+}
+
 template <int D>
 __global__ void __launch_bounds__(COMBINE_ROWS * (D / 8))
 combine_kernel(const CombineEntry* entries, const CellGeom* cells, const float* part_o, const float2* part_ml,
@@ -645,21 +653,104 @@ combine_kernel(const CombineEntry* entries, const CellGeom* cells, const float* 
   const int r = (blockIdx.x % (128 / COMBINE_ROWS)) * COMBINE_ROWS + threadIdx.x / CHUNKS;
   const int c = threadIdx.x % CHUNKS;
   if (r >= e.q_count) return;
+  // Rows of successive parts lie 256 rows apart.  The parts are taken four at a time with all loads of a batch issued
+  // before the first use (a thread has only 32 bytes per part to fetch, so one part at a time leaves the kernel waiting
+  // on one memory round trip after the other); the partial results are read once, hence the streaming loads.
+  const size_t row0 = static_cast<size_t>(e.first_slot) * 256 + e.sub * 128 + r;
+  const int n = e.n_parts;
   float m = -INFINITY;
-  for (int i = 0; i < e.n_parts; ++i)
-    m = fmaxf(m, part_ml[static_cast<size_t>(e.first_slot + i) * 256 + e.sub * 128 + r].x);
+  for (int i0 = 0; i0 < n; i0 += 4) {
+    float mk[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k)
+      mk[k] = (i0 + k < n) ? __ldg(&part_ml[row0 + static_cast<size_t>(i0 + k) * 256]).x : -INFINITY;
+    m = fmaxf(fmaxf(m, fmaxf(mk[0], mk[1])), fmaxf(mk[2], mk[3]));
+  }
   float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0}, l = 0.f;
-  for (int i = 0; i < e.n_parts; ++i) {
-    const size_t row = static_cast<size_t>(e.first_slot + i) * 256 + e.sub * 128 + r;
-    const float2 ml = part_ml[row];
+  for (int i0 = 0; i0 < n; i0 += 4) {
+    float2 ml[4];
+    float4 a[4], b[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const size_t row = row0 + static_cast<size_t>(min(i0 + k, n - 1)) * 256;  // past the end: a valid row, weight 0
+      ml[k] = __ldg(&part_ml[row]);
+      const float4* src = reinterpret_cast<const float4*>(part_o + row * D + c * 8);
+      a[k] = ld_stream_f4(src);
+      b[k] = ld_stream_f4(src + 1);
+    }
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const float wgt = (i0 + k >= n || ml[k].x == -INFINITY) ? 0.f : ex2_approx(ml[k].x - m);
+      l += wgt * ml[k].y;
+      acc[0] += wgt * a[k].x; acc[1] += wgt * a[k].y; acc[2] += wgt * a[k].z; acc[3] += wgt * a[k].w;
+      acc[4] += wgt * b[k].x; acc[5] += wgt * b[k].y; acc[6] += wgt * b[k].z; acc[7] += wgt * b[k].w;
+    }
+  }
+  const float inv = l > 0.f ? 1.f / l : 0.f;
+  int token = e.q_start + r;
+  if (e.cell >= 0) token = cell_query_token(cells[e.cell], token, tokens_per_frame, grid_w);
+  uint4 o4;
+  o4.x = pack_bf16x2(acc[0] * inv, acc[1] * inv);
+  o4.y = pack_bf16x2(acc[2] * inv, acc[3] * inv);
+  o4.z = pack_bf16x2(acc[4] * inv, acc[5] * inv);
+  o4.w = pack_bf16x2(acc[6] * inv, acc[7] * inv);
+  *reinterpret_cast<uint4*>(out + (static_cast<size_t>(token) * n_heads + e.head) * D + c * 8) = o4;
+}
+
+// The same merge for query tiles that were cut into MANY pieces (the pieces of one pair in the shared queue of the
+// dynamic tail can run to dozens): one block per ROW, the parts dealt over COMBINE_LANES groups of threads that each
+// merge their share as above, then one group merges the groups' results through shared memory.  With one thread
+// walking all parts of its row the launch ended with a few blocks each waiting on twenty memory round trips in turn.
+constexpr int COMBINE_LANES = 16;
+constexpr int COMBINE_LONG_PARTS = 16;  // entries with more parts than this go through combine_long_kernel
+
+template <int D>
+__global__ void __launch_bounds__(COMBINE_LANES * (D / 8))
+combine_long_kernel(const CombineEntry* entries, const CellGeom* cells, const float* part_o, const float2* part_ml,
+                    __nv_bfloat16* out, int n_heads, int tokens_per_frame, int grid_w) {
+  constexpr int CHUNKS = D / 8;
+  __shared__ float sh_m[COMBINE_LANES], sh_l[COMBINE_LANES];
+  __shared__ float sh_acc[COMBINE_LANES][D];
+  const CombineEntry e = entries[blockIdx.x / 128];
+  const int r = blockIdx.x % 128;
+  if (r >= e.q_count) return;  // the whole block leaves: no barrier is missed
+  const int c = threadIdx.x % CHUNKS, lane = threadIdx.x / CHUNKS;
+  const size_t row0 = static_cast<size_t>(e.first_slot) * 256 + e.sub * 128 + r;
+  const int n = e.n_parts;
+  float m = -INFINITY;
+  for (int i = lane; i < n; i += COMBINE_LANES) m = fmaxf(m, __ldg(&part_ml[row0 + static_cast<size_t>(i) * 256]).x);
+  float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0}, l = 0.f;
+  for (int i = lane; i < n; i += COMBINE_LANES) {
+    const size_t row = row0 + static_cast<size_t>(i) * 256;
+    const float2 ml = __ldg(&part_ml[row]);
+    const float4* src = reinterpret_cast<const float4*>(part_o + row * D + c * 8);
+    const float4 a = ld_stream_f4(src), b = ld_stream_f4(src + 1);
     const float wgt = (ml.x == -INFINITY) ? 0.f : ex2_approx(ml.x - m);
     l += wgt * ml.y;
-    const float4* src = reinterpret_cast<const float4*>(part_o + row * D + c * 8);
-    const float4 a = src[0], b = src[1];
     acc[0] += wgt * a.x; acc[1] += wgt * a.y; acc[2] += wgt * a.z; acc[3] += wgt * a.w;
     acc[4] += wgt * b.x; acc[5] += wgt * b.y; acc[6] += wgt * b.z; acc[7] += wgt * b.w;
   }
-  const float inv = l > 0.f ? 1.f / l : 0.f;
+  if (c == 0) {
+    sh_m[lane] = m;
+    sh_l[lane] = l;
+  }
+#pragma unroll
+  for (int k = 0; k < 8; ++k) sh_acc[lane][c * 8 + k] = acc[k];
+  __syncthreads();
+  if (lane != 0) return;
+  float m_all = -INFINITY;
+#pragma unroll
+  for (int g = 0; g < COMBINE_LANES; ++g) m_all = fmaxf(m_all, sh_m[g]);
+  float l_all = 0.f;
+#pragma unroll
+  for (int k = 0; k < 8; ++k) acc[k] = 0.f;
+  for (int g = 0; g < COMBINE_LANES; ++g) {
+    const float wgt = (sh_m[g] == -INFINITY) ? 0.f : ex2_approx(sh_m[g] - m_all);
+    l_all += wgt * sh_l[g];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) acc[k] += wgt * sh_acc[g][c * 8 + k];
+  }
+  const float inv = l_all > 0.f ? 1.f / l_all : 0.f;
   int token = e.q_start + r;
   if (e.cell >= 0) token = cell_query_token(cells[e.cell], token, tokens_per_frame, grid_w);
   uint4 o4;

@@ -50,12 +50,13 @@ struct Schedule {
   int key_filled = -1;  // cache fill the lists were built for
   std::vector<WorkItem> items;
   std::vector<int32_t> cta_first;
-  std::vector<CombineEntry> combine;
+  std::vector<CombineEntry> combine;       // query tiles to merge, up to COMBINE_LONG_PARTS pieces each
+  std::vector<CombineEntry> combine_long;  // those cut into more pieces (combine_long_kernel)
   std::vector<ClsGroup> cls_groups;  // classification only: key ranges of one query pair, merged three ways
   std::vector<ClsPart> cls_parts;
   DevBuf<WorkItem> items_dev;
   DevBuf<int32_t> cta_first_dev;
-  DevBuf<CombineEntry> combine_dev;
+  DevBuf<CombineEntry> combine_dev, combine_long_dev;
   DevBuf<ClsGroup> cls_groups_dev;
   DevBuf<ClsPart> cls_parts_dev;
   int n_slots = 0;
@@ -66,6 +67,7 @@ struct Schedule {
     items_dev.release();
     cta_first_dev.release();
     combine_dev.release();
+    combine_long_dev.release();
     cls_groups_dev.release();
     cls_parts_dev.release();
   }
@@ -297,6 +299,7 @@ double item_cost(const WorkItem& w) {
 void finalize_schedule(headcast_ctx* c, Schedule& s, std::vector<Proto>& protos, bool allow_split) {
   s.items.clear();
   s.combine.clear();
+  s.combine_long.clear();
   s.n_slots = 0;
   const int n_cta = c->n_sm;
   std::vector<std::vector<WorkItem>> bins(n_cta + 1);  // bins[n_cta]: the shared queue (dynamic tail)
@@ -584,6 +587,7 @@ void finalize_schedule(headcast_ctx* c, Schedule& s, std::vector<Proto>& protos,
           by_group[w.out_slot].push_back({b, static_cast<int>(i), w.tile_begin});
         }
       s.combine.clear();
+      s.combine_long.clear();
       s.n_slots = 0;
       for (auto& pieces : by_group) {
         if (pieces.empty()) continue;
@@ -607,7 +611,7 @@ void finalize_schedule(headcast_ctx* c, Schedule& s, std::vector<Proto>& protos,
           e.n_parts = static_cast<int32_t>(pieces.size());
           e.sub = t;
           e.pad = 0;
-          s.combine.push_back(e);
+          (e.n_parts > COMBINE_LONG_PARTS ? s.combine_long : s.combine).push_back(e);
         }
       }
     }
@@ -711,6 +715,11 @@ int upload_schedule(headcast_ctx* c, Schedule& s, cudaStream_t st) {
   if (!s.combine.empty())
     HC_CUDA(c, cudaMemcpyAsync(s.combine_dev.ptr, s.combine.data(), s.combine.size() * sizeof(CombineEntry),
                                cudaMemcpyHostToDevice, st));
+  if (!s.combine_long.empty()) {
+    HC_CUDA(c, s.combine_long_dev.reserve(s.combine_long.size()));
+    HC_CUDA(c, cudaMemcpyAsync(s.combine_long_dev.ptr, s.combine_long.data(), s.combine_long.size() * sizeof(CombineEntry),
+                               cudaMemcpyHostToDevice, st));
+  }
   if (!s.cls_groups.empty()) {
     HC_CUDA(c, s.cls_groups_dev.reserve(s.cls_groups.size()));
     HC_CUDA(c, s.cls_parts_dev.reserve(std::max<size_t>(1, s.cls_parts.size())));
@@ -832,6 +841,17 @@ int run_schedule(headcast_ctx* c, Schedule& s, const void* q, void* out, bool pr
     else
       combine_kernel<64><<<blocks, COMBINE_ROWS * 8, 0, st>>>(s.combine_dev.ptr, c->cells_dev, c->part_o.ptr,
                                                               c->part_ml.ptr, p.out, c->H, c->T_f, c->G_w);
+    HC_CUDA(c, cudaGetLastError());
+    ++c->launches;
+  }
+  if (!s.combine_long.empty()) {
+    const unsigned blocks = static_cast<unsigned>(s.combine_long.size()) * 128;  // one block per query row
+    if (c->D == 128)
+      combine_long_kernel<128><<<blocks, COMBINE_LANES * 16, 0, st>>>(s.combine_long_dev.ptr, c->cells_dev, c->part_o.ptr,
+                                                                      c->part_ml.ptr, p.out, c->H, c->T_f, c->G_w);
+    else
+      combine_long_kernel<64><<<blocks, COMBINE_LANES * 8, 0, st>>>(s.combine_long_dev.ptr, c->cells_dev, c->part_o.ptr,
+                                                                     c->part_ml.ptr, p.out, c->H, c->T_f, c->G_w);
     HC_CUDA(c, cudaGetLastError());
     ++c->launches;
   }

@@ -105,8 +105,9 @@ def check_plan(w, labels, n_filled, n_ctas, dense=False):
     # small part of the launch, in pieces small enough that the last one drawn cannot delay the end by much
     queue = cost[first[-1]:]
     if queue.size:
-        # (2 % of the launch by design, plus the cost of the cuts that the equal static shares did not allow for)
-        assert queue.sum() <= 0.08 * cost.sum() + 40.0
+        # (2 % of the launch by design, plus the cost of the cuts that the equal static shares did not allow for, which
+        # weighs more the shorter the launch)
+        assert queue.sum() <= (0.08 if cost.sum() > 200.0 * n_ctas else 0.15) * cost.sum() + 40.0
         q_tiles = (items[first[-1]:, F["tile_end"]] - items[first[-1]:, F["tile_begin"]]).max()
         assert q_tiles <= max(8, 0.02 * cost.sum() / (4 * n_ctas)) + 4  # a piece, plus a remainder too short to stand alone
     return items, per_cta
