@@ -744,6 +744,33 @@ def test_contexts_give_their_device_memory_back():
     assert in_use() - before < 8.0
 
 
+def test_query_tiles_cut_into_dozens_of_pieces_are_merged_row_by_row():
+    """Six Global heads over a 32-block window at a 32x32 grid: the launch is long enough for the shared queue at its
+    end, whose pieces are cuts of the last pairs - those pairs end up in about thirty pieces each, which the merge
+    handles with one block per row.  The host plan says which rows those are; they are all compared."""
+    w = synth.Workload(name="long_groups", n_heads=6, head_dim=128, grid_h=32, grid_w=32, n_blocks=32,
+                       frames_per_block=1, cell_h=8, cell_w=8, labels=(orc.GLOBAL,) * 6, seed=synth.BASE_SEED + 321)
+    from paper_2607_20125_b200 import binding
+    from test_schedule_host import F, config_of
+    items, first = binding.plan_schedule(config_of(w), list(w.labels), w.n_blocks, 148)
+    parts = {}
+    for it in items:
+        if it[F["out_mode"]] == 1:
+            key = (int(it[F["head"]]), int(it[F["q_start0"]]))
+            parts[key] = parts.get(key, 0) + 1
+    long_pairs = [k for k, n in parts.items() if n > 16]
+    assert long_pairs and first[-1] < len(items), "the plan no longer has a pair in more than 16 pieces: pick another shape"
+    rows = np.unique(np.concatenate([np.arange(q0, min(q0 + 256, w.block_tokens), 5) for _, q0 in long_pairs]
+                                    + [np.arange(0, w.block_tokens, 37)]))
+    p = Pair(w)
+    p.append(w.n_blocks)
+    p.hc.set_labels(w.labels)
+    p.hc.split_cache()
+    p.cache.split(w.labels)
+    p.check_attention(dense=False, rows=rows)
+    p.check_attention(dense=True, rows=rows)
+
+
 @pytest.mark.parametrize("scale", [0.01, 16.0, 256.0])
 def test_flat_peaked_and_huge_logits(scale):
     # queries scaled so that the softmax is nearly uniform, nearly one-hot, or has logits in the thousands; a few rows
