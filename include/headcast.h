@@ -21,7 +21,9 @@
  *     headcast_create / headcast_split_cache and frees at headcast_destroy).  The caller must
  *     keep the context's device current and must not use one context from two threads at once.
  *   - a kernel that gave up on a bounded wait sets a device status word; the next synchronising
- *     call, or headcast_check(), reports it as HC_ERR_TIMEOUT.
+ *     call, or headcast_check(), reports it as HC_ERR_TIMEOUT.  Until it has been reported, later
+ *     attention launches of the context return at once without computing anything (their
+ *     outputs are undefined); reading the status clears it and puts the context back to work.
  *
  * States: FILLING (monolithic cache only) --headcast_split_cache--> SPLIT.  A call made in
  * the wrong state returns HC_ERR_STATE and changes nothing.

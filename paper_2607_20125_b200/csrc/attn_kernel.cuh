@@ -170,7 +170,10 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const __grid_cons
       mbar_init(&bar_kv_free[s], 1);
     }
     for (int s = 0; s < 4; ++s) mbar_init(&bar_dyn[s], 1);
-    abort_flag = 0;
+    // A context whose earlier kernel gave up on a wait keeps its status word set until the host has read it; the
+    // shared queue's counters may then be half drawn, so until then a launch does nothing at all (every thread sees
+    // the same answer: one thread reads the word, the others read its copy after the barrier below)
+    abort_flag = (*reinterpret_cast<volatile int32_t*>(p.status) != 0) ? 1 : 0;
     fence_mbar_init();
   }
   if (warp == 1) {
@@ -183,6 +186,7 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const __grid_cons
   const uint32_t tmem = tmem_slot;
   volatile int* abortp = &abort_flag;
 
+  const bool dead_on_arrival = abort_flag != 0;  // read before any wait of this launch can raise the flag
   const int item_lo = p.cta_first[blockIdx.x], item_hi = p.cta_first[blockIdx.x + 1];
   const bool has_queue = p.dyn_end > p.dyn_first;
   // Items come from the CTA's own list first, then from the shared queue.  The producer thread draws the queue
@@ -221,8 +225,9 @@ __global__ void __launch_bounds__(ATTN_THREADS, 1) attn_kernel(const __grid_cons
     return v >= 0;
   };
 
-
-  if (warp == 0) {
+  if (dead_on_arrival) {
+    // nothing: straight to the teardown
+  } else if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
       uint32_t kt = 0;
