@@ -992,8 +992,7 @@ int launch_move(headcast_ctx* c, const RouteParams& r, int n_src, cudaStream_t s
   if (jobs == 0) return HC_OK;
   if (jobs >= (1ll << 31)) return fail(c, HC_ERR_UNSUPPORTED, "too many tile jobs");
   const int ctas = static_cast<int>(std::min<long long>(c->n_sm, (jobs + MOVE_ENGINES - 1) / MOVE_ENGINES));
-  cudaLaunchConfig_t lc;
-  std::memset(&lc, 0, sizeof(lc));
+  cudaLaunchConfig_t lc = {};
   lc.gridDim = dim3(ctas);
   lc.blockDim = dim3(MOVE_ENGINES * 32);
   lc.dynamicSmemBytes = MOVE_SMEM_BYTES;
@@ -1665,7 +1664,7 @@ int headcast_export_cache(headcast_ctx* c, int32_t head, void* k_out, void* v_ou
   e.frames_per_block = c->F_b;
   e.n_blocks = c->n_blk;
   e.sd_slots = c->sd_slots;
-  const int cl = (c->state == STATE_SPLIT) ? c->cls[head] : CLS_NONE;
+  const int cl = (c->state == STATE_SPLIT) ? static_cast<int>(c->cls[head]) : static_cast<int>(CLS_NONE);
   if (cl == CLS_NONE) {
     e.layout = 0; e.head = head; e.src_k = reinterpret_cast<const uint4*>(c->mono_k); e.src_v = reinterpret_cast<const uint4*>(c->mono_v);
   } else if (cl == CLS_GLOBAL) {
