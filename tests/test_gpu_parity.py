@@ -744,6 +744,29 @@ def test_contexts_give_their_device_memory_back():
     assert in_use() - before < 8.0
 
 
+def test_repeated_attends_are_bit_identical_with_the_shared_queue():
+    """At 480P the end of a launch is drawn from the shared queue by whichever CTA is free: which CTA runs a piece changes
+    from launch to launch, what it computes and the order of the merge do not, so repeated calls give the same bits."""
+    import torch
+    w = synth.wan("480p")
+    from paper_2607_20125_b200 import binding
+    from test_schedule_host import config_of
+    items, first = binding.plan_schedule(config_of(w), list(w.labels), w.n_blocks, 148)
+    assert first[-1] < len(items), "no shared queue at this size any more: pick a larger one"
+    p = Pair(w)
+    p.append(w.n_blocks)
+    p.hc.set_labels(w.labels)
+    p.hc.split_cache()
+    q = to_dev(synth.make_q(w, w.n_blocks - 1, 0))
+    ref = torch.empty((w.block_tokens, w.n_heads, w.head_dim), dtype=torch.bfloat16, device="cuda")
+    p.hc.attend(q, ref)
+    outs = [torch.full_like(ref, float("nan")) for _ in range(8)]
+    for rep in range(40):
+        p.hc.attend(q, outs[rep % 8])
+    p.hc.check()
+    assert all(torch.equal(o, ref) for o in outs)
+
+
 def test_query_tiles_cut_into_dozens_of_pieces_are_merged_row_by_row():
     """Six Global heads over a 32-block window at a 32x32 grid: the launch is long enough for the shared queue at its
     end, whose pieces are cuts of the last pairs - those pairs end up in about thirty pieces each, which the merge
